@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the ESPO hot path on B200: fused decode step (rows/s, GB/s vs HBM peak) + advantage pass.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A timed "step" is one espo_step call over the rollout batch (B=512 trajectories x V=152064
+bf16 logits, temperature 1: the paper's 64 prompts x 8 rollouts at a Qwen-sized vocabulary).
+The timed region is a rollout of K such steps followed by ONE espo_advantages pass over the
+K*B tokens that rollout generated -- the whole path, at the cadence the method runs it.
+The advantage kernel is additionally timed on its own workload (1024 ragged trajectories of
+256..16384 tokens) and reported under "advantage_pass".
+
+Prints one JSON line (see the design doc for the field-by-field definition).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+B_ROWS = 512
+VOCAB = 152064
+N_BUFFERS = 4                 # 4 x 155.7 MB of logits rotate, so no step finds its rows in the 126 MB L2
+ADV_B = 1024
+TRAFFIC_STEP_BYTES = None     # dram bytes per launch from an ncu capture of the step kernel (profiles/), if any
+
+PARAMS = dict(temperature=1.0, mu_g=6.0, sigma2_g=9.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0, eps=0.2,
+              warmup_complete=1, t_max=1 << 30, eos_token=-1)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50", "-i", str(self.gpu)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+
+        def pump():
+            for line in self.proc.stdout:
+                self.rows.append((time.time(), line.strip()))
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()       # the exact process started above
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self, t0: float, t1: float) -> dict:
+        def parse(rows):
+            sm, mx, reasons = [], [], set()
+            for _, line in rows:
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0])); mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            return sm, mx, reasons
+        inside = [r for r in self.rows if t0 <= r[0] <= t1]
+        window = "timed region"
+        if not inside:
+            inside, window = self.rows, "whole run (timed region shorter than the sampling period)"
+        sm, mx, reasons = parse(inside)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "nvidia-smi unavailable"}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "window": window}
+
+
+def cpu_threads() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_step_rate(rows_f32, values, seconds_target: float, sampler: int):
+    """Time the CPU oracle (as it stands) on a bounded sample of the benchmark's rows; returns rows/s.
+
+    The sample rows are advanced decode step after decode step (new draws each step) on all host
+    cores until about `seconds_target` seconds have passed.
+    """
+    import oracle
+    cores = cpu_threads()
+    p = oracle.make_params(sampler=sampler, **PARAMS)
+    n = rows_f32.shape[0]
+    ro = oracle.Rollout(n, seed=1)
+    done, t0 = 0, time.perf_counter()
+    while True:
+        ro.step_f32(rows_f32, values, p, n_threads=cores)
+        done += n
+        dt = time.perf_counter() - t0
+        if dt >= seconds_target:
+            break
+    return done / dt, cores, done, dt
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, same metric and config, bounded sample per step."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2605_29860_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = cpu_threads()
+    sample_rows = 32
+    x = synth.logits_batch(sample_rows, VOCAB, dtype=torch.bfloat16, sd=3.0, seed=100, device="cpu").float().numpy()
+    vals = np.full(sample_rows, 0.5)
+    p = oracle.make_params(sampler=oracle.SAMPLER_HIER, **PARAMS)
+    ro = oracle.Rollout(sample_rows, seed=1)
+    for _ in range(args.warmup):
+        ro.step_f32(x, vals, p, n_threads=cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ro.step_f32(x, vals, p, n_threads=cores)
+    dt = time.perf_counter() - t0
+    value = sample_rows * args.steps / dt
+    sample = f"{sample_rows} rows of the {B_ROWS}x{VOCAB} bf16 batch per step, hierarchical sampler"
+    print(json.dumps({
+        "impl": "reference", "metric": "fused ESPO step logit rows/s at V=152064 bf16", "value": value, "unit": "rows/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"rollout-batch scale: B={B_ROWS}, V={VOCAB}, bf16 logits, temperature 1.0 "
+                               f"(CPU oracle on a {sample_rows}-row sample per step)"},
+        "cpu_baseline": {"value": value, "unit": "rows/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "rows/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows", type=int, default=B_ROWS, help="rollout batch size B (default: the headline 512)")
+    ap.add_argument("--sampler", default="hier", choices=["hier", "flat"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = args.steps or 4
+        args.warmup = args.warmup if args.warmup is not None else 1
+        return run_reference(args)
+    args.steps = args.steps or 20000
+    args.warmup = max(3, args.warmup if args.warmup is not None else 200)
+
+    import numpy as np
+    import torch
+    import paper_2605_29860_b200 as espo
+    from paper_2605_29860_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+
+    B, V, K, W = args.rows, VOCAB, args.steps, args.warmup
+    sampler = espo.ESPO_SAMPLER_HIER if args.sampler == "hier" else espo.ESPO_SAMPLER_FLAT
+    params = espo.make_params(sampler=sampler, **PARAMS)
+    # ---- synthetic inputs, resident in HBM: every rank owns its own B rows (rows are independent) ----
+    bufs = [synth.logits_batch(B, V, dtype=torch.bfloat16, sd=3.0, seed=100 + 10 * rank + i, device=dev)
+            for i in range(N_BUFFERS)]
+    values = torch.full((B,), 0.5, dtype=torch.bfloat16, device=dev)
+    tokens = torch.empty(B, dtype=torch.int32, device=dev)
+    stop = torch.empty(B, dtype=torch.uint8, device=dev)
+    state = espo.espo_init_state(B, V, seed=1234 + rank)
+    view = espo.espo_state_view(state)
+    # rollout record for the closing advantage pass: K tokens per trajectory, reward 0 except the end
+    adv_tokens = B * K
+    adv_r = torch.zeros(adv_tokens, device=dev)
+    adv_v = torch.full((adv_tokens,), 0.5, device=dev)
+    adv_out = torch.empty(adv_tokens, device=dev)
+    adv_len = torch.full((B,), K, dtype=torch.int32, device=dev)
+    adv_stopped = torch.zeros(B, dtype=torch.uint8, device=dev)
+    espo.espo_advantages_reserve(max(B, ADV_B), max(adv_tokens, ADV_B * 16384))
+
+    def rollout(n_steps):
+        for i in range(n_steps):
+            espo.espo_step(bufs[i % N_BUFFERS], values, state, params, tokens, stop)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    rollout(W)
+    espo.espo_advantages(adv_r, adv_v, adv_len, adv_stopped, 1.0, 0.95, -1.0, adv_out)
+    espo.espo_reset_state(state, 0)
+    sampler_proc = ClockSampler(local_rank) if rank == 0 else None
+    if sampler_proc:
+        sampler_proc.start()
+        time.sleep(0.3)
+    barrier()
+    ev0, ev1, ev2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    t_wall0 = time.time()
+    ev0.record()
+    rollout(K)
+    ev1.record()
+    espo.espo_advantages(adv_r, adv_v, adv_len, adv_stopped, 1.0, 0.95, -1.0, adv_out)
+    ev2.record()
+    barrier()
+    t_wall1 = time.time()
+    ms_total = ev0.elapsed_time(ev2)
+    ms_steps = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms_total, ms_steps], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_steps = t.tolist()
+    if sampler_proc:
+        time.sleep(0.1)
+        sampler_proc.stop()
+    dev_status = espo.espo_state_status(state) | espo.espo_advantages_status()
+    n_stopped = int((view["status"] != espo.ESPO_ROW_ACTIVE).sum().item())
+    assert int(view["t"].min().item()) == K or n_stopped > 0, "the timed rollout did not advance every trajectory"
+
+    rows_per_s = world * B * K / (ms_total * 1e-3)
+    bytes_per_launch = B * V * 2
+    kernel_ms = ms_steps / K
+    peak, peak_kind = measured_peaks()
+    achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
+
+    out = {
+        "metric": "fused ESPO step logit rows/s at V=152064 bf16", "value": rows_per_s, "unit": "rows/s",
+        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": f"rollout-batch scale: B={B} trajectories per GPU, V={V}, bf16 logits ~N(0,3) + 5 Zipf peaks, "
+                        f"temperature 1.0, {args.sampler} Philox Gumbel-max sampler, full active set; timed region = "
+                        f"{K} decode steps + 1 advantage pass over the {adv_tokens} tokens generated",
+            "l2": f"{N_BUFFERS} logit buffers of {bytes_per_launch / 1e6:.1f} MB rotate (each larger than the 126 MB L2)",
+            "parallelism": f"rows sharded over {world} GPU(s), no collective",
+            "stopped_rows": n_stopped, "device_status": dev_status,
+        },
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": TRAFFIC_STEP_BYTES, "kernel": "espo_step_kernel<bf16,hier,bulk>",
+                     "peak_kind": f"of {peak_kind} copy bandwidth", "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "launch_us": kernel_ms * 1e3, "bytes_per_launch": bytes_per_launch},
+        "gpu_launches": K + 2,
+    }
+
+    if rank == 0:
+        # ---- the advantage kernel on its own workload (ragged batch of 1024 trajectories) ----
+        r, v, L, s = synth.ragged_trajectories(ADV_B, seed=0, device=dev)
+        a_out = torch.empty_like(r)
+        n_tok = r.numel()
+        for lam in (0.95,):
+            for _ in range(5):
+                espo.espo_advantages(r, v, L, s, 1.0, lam, -1.0, a_out)
+            torch.cuda.synchronize()
+            reps = 50
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                espo.espo_advantages(r, v, L, s, 1.0, lam, -1.0, a_out)
+            e1.record()
+            torch.cuda.synchronize()
+            adv_ms = e0.elapsed_time(e1) / reps
+        adv_gbs = 12.0 * n_tok / (adv_ms * 1e-3) / 1e9
+        out["advantage_pass"] = {
+            "workload": f"B={ADV_B} ragged trajectories, lengths U[256,16384] ({n_tok} tokens, "
+                        f"{12.0 * n_tok / 1e6:.1f} MB of traffic > L2), 35% stopped, gamma=1, lambda=0.95",
+            "tokens_per_s": n_tok / (adv_ms * 1e-3), "ms": adv_ms,
+            "roofline": {"bound": "hbm", "achieved": adv_gbs, "peak": peak, "unit": "GB/s", "frac": adv_gbs / peak,
+                         "traffic": None, "bytes_per_token": 12},
+        }
+        del r, v, L, s, a_out
+
+        # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region ----
+        host_logits = [torch.empty(B, V, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+        for i in range(2):
+            host_logits[i].copy_(bufs[i])
+        host_values = torch.full((B,), 0.5, dtype=torch.bfloat16).pin_memory()
+        host_tokens = torch.empty(B, dtype=torch.int32).pin_memory()
+        host_stop = torch.empty(B, dtype=torch.uint8).pin_memory()
+        dev_logits = torch.empty(B, V, dtype=torch.bfloat16, device=dev)
+        dev_values = torch.empty(B, dtype=torch.bfloat16, device=dev)
+        espo.espo_reset_state(state, 1)
+
+        def e2e_step(i):
+            dev_logits.copy_(host_logits[i % 2], non_blocking=True)
+            dev_values.copy_(host_values, non_blocking=True)
+            espo.espo_step(dev_logits, dev_values, state, params, tokens, stop)
+            host_tokens.copy_(tokens, non_blocking=True)
+            host_stop.copy_(stop, non_blocking=True)
+            torch.cuda.synchronize()       # the caller needs the tokens before the next decode step
+
+        for i in range(3):
+            e2e_step(i)
+        n_e2e = 20
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            e2e_step(i)
+        dt = time.perf_counter() - t0
+        out["e2e"] = {"value": B * n_e2e / dt, "unit": "rows/s", "h2d_bytes_per_step": B * V * 2 + B * 2,
+                      "d2h_bytes_per_step": B * 4 + B, "steps": n_e2e, "n_gpus": 1,
+                      "note": "pinned host logits copied in, tokens and stop mask copied out, every step"}
+        del host_logits, dev_logits
+
+        # ---- clocks ----
+        out["clocks"] = sampler_proc.summary(t_wall0, t_wall1) if sampler_proc else None
+
+        # ---- the CPU oracle on this machine's host cores, on a bounded sample of the same rows ----
+        if not args.no_cpu_baseline:
+            sample_src = bufs[0][:256].float().cpu().numpy()
+            rate, cores, n_rows, secs = oracle_step_rate(sample_src, np.full(256, 0.5), 12.0, sampler)
+            out["cpu_baseline"] = {"value": rate, "unit": "rows/s", "cores": cores, "kind": "oracle",
+                                   "sample": f"{n_rows} row-steps: rows 0..255 of buffer 0 advanced step after step "
+                                             f"for {secs:.1f} s on {cores} threads"}
+        print(json.dumps(out))
+    espo.espo_free_state(state)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,202 @@
+/* espo.h -- C ABI of the ESPO early-stopping hot path for NVIDIA B200 (sm_100a).
+ *
+ * ESPO (Early-Stopping Proximal Policy Optimization) ends a rollout during decoding
+ * once a smoothed, normalised regret signal computed from the policy's own logits
+ * exceeds a threshold gated by the critic's value estimate, and trains on the
+ * truncated prefix as an absorbing failure transition.  This library implements the
+ * two data-parallel pieces of that method:
+ *
+ *   espo_step        one pass of the rollout loop body (Algorithm 1) over a batch of
+ *                    logit rows: log-softmax statistics, Philox Gumbel-max sampling,
+ *                    surrogate regret (Eq. 5), normalisation (Eq. 8), smoothing (Eq. 9),
+ *                    value-gated stop test (Eq. 10), per-trajectory bookkeeping;
+ *   espo_advantages  TD errors and GAE (Eq. 3-4) over ragged truncated trajectories with
+ *                    the failure transition of Eq. 12.
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA device memory owned by the caller, on the device that
+ *     was current when the state was created; "host" pointers are ordinary memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
+ *     only enqueued; no entry point synchronises the host unless it says so.
+ *   - Every function returns an int: ESPO_OK (0) or a negative ESPO_ERR_* code.
+ *     Argument errors are found on the host before anything is launched.  Conditions
+ *     found on the device (unusable logit rows, bad slot ids, a wait that ran out) are
+ *     recorded in a sticky device status word, never trapped.
+ *   - There is no CPU fallback: without a CUDA device the calls return ESPO_ERR_CUDA.
+ */
+#ifndef ESPO_H_
+#define ESPO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- return codes ------------------------------------------------------------------ */
+#define ESPO_OK              0
+#define ESPO_ERR_NULL       -1   /* a required pointer was NULL                          */
+#define ESPO_ERR_BAD_DTYPE  -2   /* dtype code is not ESPO_F32 / ESPO_BF16                */
+#define ESPO_ERR_BAD_SHAPE  -3   /* a size is non-positive, or a stride is shorter than V */
+#define ESPO_ERR_ALIGN      -4   /* a pointer is not aligned to its element type          */
+#define ESPO_ERR_CAPACITY   -5   /* more rows / tokens than the state or workspace holds  */
+#define ESPO_ERR_CUDA       -6   /* a CUDA runtime call failed (see espo_last_cuda_error) */
+#define ESPO_ERR_BAD_PARAM  -7   /* a parameter is outside its documented range           */
+
+/* ---- element types of caller buffers ----------------------------------------------- */
+#define ESPO_F32   0
+#define ESPO_BF16  1
+
+/* ---- sampler ------------------------------------------------------------------------ */
+/* Both draw a_t ~ softmax(logits / temperature) exactly, by Gumbel-max with Philox4x32-10
+ * noise keyed by (seed; batch_id, trajectory slot, step, index).  They differ in how many
+ * draws they need and therefore return different (equally valid) tokens.
+ *   FLAT  one draw per vocabulary id: a_t = argmax_a (x_a + G_a).
+ *   HIER  the same argmax taken level by level -- first over blocks of 1024 ids scored by
+ *         their log-sum-exp, then over sub-blocks of 32 ids inside the winner, then over
+ *         the 32 ids -- which needs ~V/1024 + 64 draws per row instead of V.            */
+#define ESPO_SAMPLER_FLAT  0
+#define ESPO_SAMPLER_HIER  1
+
+/* ---- per-trajectory status (espo_state_view: status[]) ------------------------------ */
+#define ESPO_ROW_ACTIVE   0
+#define ESPO_ROW_STOPPED  1   /* ESPO's rule fired (Eq. 10): failure transition            */
+#define ESPO_ROW_EOS      2   /* sampled the end-of-sequence token                          */
+#define ESPO_ROW_TMAX     3   /* reached the horizon t_max                                  */
+#define ESPO_ROW_BAD      4   /* the logit row held NaN / +inf, or no finite entry          */
+
+/* ---- bits of the sticky device status word (espo_state_status) ---------------------- */
+#define ESPO_DEV_BAD_ROW     1u   /* some row was marked ESPO_ROW_BAD                       */
+#define ESPO_DEV_BAD_SLOT    2u   /* a row_ids entry was outside [0, capacity)              */
+#define ESPO_DEV_TIMEOUT     4u   /* a bounded in-kernel wait ran out; results incomplete   */
+#define ESPO_DEV_NAN_VALUE   8u   /* a value estimate was NaN (that row did not stop)       */
+#define ESPO_DEV_BAD_LENGTHS 16u  /* espo_advantages: sum(lengths) != total_tokens or L < 0 */
+
+/* Parameters that stay frozen for a whole rollout batch (Sec. 4.2: the statistics are
+ * only updated at batch boundaries).  Plain data, passed by host pointer, copied at call. */
+typedef struct espo_params {
+  float   temperature;      /* > 0 samples from softmax(logits/temperature); 0 = greedy    */
+  float   mu_g;             /* running mean of the regret, Eq. 6                            */
+  float   sigma2_g;         /* running variance of the regret, Eq. 7 (>= 0)                 */
+  float   delta;            /* stabiliser under the square root in Eq. 8 (sigma2_g+delta>0) */
+  float   clip_c;           /* clipping bound c of Eq. 8 (> 0)                              */
+  float   alpha_s;          /* smoothing factor of Eq. 9, in [0, 1)                         */
+  float   beta;             /* threshold multiplier of Eq. 10                               */
+  float   eps;              /* value floor epsilon of Eq. 10                                */
+  int32_t warmup_complete;  /* 0: the stop test is disabled (critic warm-up); z still runs  */
+  int32_t t_max;            /* horizon T_max (> 0)                                          */
+  int32_t eos_token;        /* end-of-sequence id, or -1 for none                           */
+  int32_t sampler;          /* ESPO_SAMPLER_FLAT or ESPO_SAMPLER_HIER                       */
+} espo_params;
+
+/* Opaque per-rollout-batch state: for each of `capacity` trajectory slots the smoothed
+ * regret z, the step counter t, the status, and running sums of g; plus the library's
+ * scratch.  Created and destroyed by the library; lives on the device current at creation. */
+typedef struct espo_state espo_state;
+
+/* Create the state for up to `capacity` trajectories over a vocabulary of V ids
+ * (Algorithm 1, line 1: z = 0, t = 0, not done -- for every slot).
+ *   out       host pointer that receives the handle
+ *   seed      64-bit Philox key;  batch_id  rollout-batch number (< 2^30), part of the counter
+ * Allocates device memory (this call and espo_free_state are the only ones that do for the
+ * step path) and enqueues the initialisation on `stream`.
+ * Errors: NULL, BAD_SHAPE (capacity or V < 1), BAD_PARAM (batch_id >= 2^30), CAPACITY, CUDA. */
+int espo_init_state(espo_state** out, int32_t capacity, int32_t V, uint64_t seed, uint64_t batch_id,
+                    void* stream);
+
+/* Start a new rollout batch in an existing state: every slot back to z = 0, t = 0, active,
+ * sums cleared, sticky status cleared; new batch_id.  Enqueued on `stream`. */
+int espo_reset_state(espo_state* st, uint64_t batch_id, void* stream);
+
+/* Release the state and its device memory (synchronises the device). NULL is ignored. */
+void espo_free_state(espo_state* st);
+
+/* One decode step for n_rows trajectories (Algorithm 1, loop body; Eq. 5, 8, 9, 10).
+ *   logits      device, [n_rows, V] row-major, element type logits_dtype, rows row_stride
+ *               ELEMENTS apart (row_stride >= V).  Read exactly once from DRAM.  Entries may
+ *               be -inf (masked ids).  The fast path needs a 16-byte aligned base and
+ *               row_stride*sizeof(elem) and V*sizeof(elem) multiples of 16; anything else
+ *               takes a slower element-wise loader with identical results.
+ *   values      device, [n_rows] critic estimates V_phi(s_t) for the same positions, values_dtype
+ *   row_ids     device, [n_rows] trajectory slot of each row, or NULL for row i = slot i.
+ *               Slots must be distinct within a call.
+ *   n_rows      0 <= n_rows <= capacity (0 is a no-op)
+ *   params      host pointer; copied before the call returns
+ *   tokens_out  device int32 [n_rows]: the sampled token a_t; -1 for a row whose slot is not
+ *               active (such rows are otherwise left untouched); 0 for an unusable row
+ *   stop_out    device uint8 [n_rows]: 1 iff ESPO's rule fired for the row on this step.
+ *               EOS and T_max endings are reported through status[], not here; a sampled
+ *               EOS takes precedence over a stop on the same step.
+ * For an active row with step counter t the call draws a_t (Philox counter uses t), forms
+ * g_t = (max logit - logit[a_t]) / temperature, g~_t, z <- alpha_s z + (1-alpha_s) g~_t,
+ * adds g_t and g_t^2 to the slot's running sums, sets t <- t+1, and updates status/t_stop.
+ * mu_g, sigma2_g and beta are never modified.  Enqueued on `stream`; calls on the same
+ * state must not overlap on the device.
+ * Errors: NULL, BAD_DTYPE, BAD_SHAPE, ALIGN, CAPACITY, BAD_PARAM, CUDA. */
+int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride,
+              const void* values, int32_t values_dtype,
+              const int32_t* row_ids, int32_t n_rows,
+              espo_state* st, const espo_params* params,
+              int32_t* tokens_out, uint8_t* stop_out, void* stream);
+
+/* Read-only device pointers to the per-slot arrays (each of length capacity); any output
+ * pointer may be NULL.  g, g_tilde and logp hold the values of each slot's latest step
+ * (logp = log pi(a_t | s_t) under the temperature-scaled distribution).  t is the number
+ * of tokens generated; t_stop is the index of the stop step or -1; sum_g, sum_g2 are the
+ * double-precision sums over the slot's tokens that the batch statistics of Eq. 6-7 need. */
+int espo_state_view(espo_state* st, const float** z, const float** g, const float** g_tilde,
+                    const float** logp, const int32_t** t, const uint8_t** status,
+                    const int32_t** t_stop, const double** sum_g, const double** sum_g2);
+
+/* Expert knob: override the step kernel's launch shape for this state.  stages = number of
+ * shared-memory ring stages per CTA, ctas_per_sm = resident CTAs per SM; 0 keeps the
+ * library default for either.  Results never depend on it.  Errors: NULL, BAD_PARAM. */
+int espo_set_launch_config(espo_state* st, int32_t stages, int32_t ctas_per_sm);
+
+/* Stable compaction of the active set: writes the slots whose status is ESPO_ROW_ACTIVE, in
+ * increasing order, to row_ids_out (device int32 [capacity]) and their number to
+ * n_active_out (device int32 [1]).  Enqueued on `stream`. */
+int espo_compact_active(espo_state* st, int32_t* row_ids_out, int32_t* n_active_out, void* stream);
+
+/* Copy the sticky device status word (ESPO_DEV_* bits) to *host_out.  Synchronises `stream`. */
+int espo_state_status(espo_state* st, uint32_t* host_out, void* stream);
+
+/* TD errors and GAE over B ragged trajectories (Eq. 3-4) with ESPO's failure transition
+ * (Eq. 12).  Trajectory i owns tokens [off_i, off_i + lengths[i]) of the packed arrays,
+ * off = exclusive prefix sum of lengths.
+ *   rewards, values  device float32 [total_tokens]
+ *   lengths          device int32 [B] (>= 0; the stop-step token of a stopped trajectory is
+ *                    its last token)
+ *   stopped          device uint8 [B]: 1 = ended by ESPO's rule; its last reward is REPLACED
+ *                    by r_fail
+ *   total_tokens     host value of sum(lengths); a mismatch sets ESPO_DEV_BAD_LENGTHS
+ *   adv_out          device float32 [total_tokens]
+ * With r'_t the (possibly replaced) rewards and V_L := 0 for every trajectory (nothing is
+ * bootstrapped past the last token): delta_t = r'_t + gamma V_{t+1} - V_t and
+ * A_t = delta_t + gamma*lambda*A_{t+1}, A_L := 0.
+ * Uses a per-device workspace that grows on demand: a call that needs more than any
+ * earlier call (or espo_advantages_reserve) allocates device memory after synchronising
+ * the device; otherwise nothing is allocated.  Calls on one device must not overlap.
+ * Errors: NULL, BAD_SHAPE, ALIGN (arrays must be 16-byte aligned), CUDA. */
+int espo_advantages(const float* rewards, const float* values, const int32_t* lengths,
+                    const uint8_t* stopped, int32_t B, int64_t total_tokens,
+                    float gamma, float lambda, float r_fail, float* adv_out, void* stream);
+
+/* Pre-size the advantage workspace of the current device so that later calls with
+ * B <= max_B and total_tokens <= max_tokens allocate nothing. */
+int espo_advantages_reserve(int32_t max_B, int64_t max_tokens);
+
+/* Copy the advantage workspace's sticky status word (ESPO_DEV_TIMEOUT, ESPO_DEV_BAD_LENGTHS)
+ * of the current device to *host_out and clear it.  Synchronises `stream`. */
+int espo_advantages_status(uint32_t* host_out, void* stream);
+
+/* Text for a return code; never NULL. */
+const char* espo_strerror(int code);
+
+/* The last cudaError_t (as int) seen by this library on the calling thread, 0 if none. */
+int espo_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ESPO_H_ */

@@ -1,0 +1,239 @@
+"""Thin ctypes binding over ``libespo.so``: same names as the C ABI, argument marshalling only.
+
+Every step of the method runs inside the CUDA library.  PyTorch is used here only to hold
+device memory and to name the current stream.  There is no CPU fallback: if the shared
+library is missing or no CUDA device is present the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+ESPO_OK = 0
+ESPO_ERR_NULL, ESPO_ERR_BAD_DTYPE, ESPO_ERR_BAD_SHAPE, ESPO_ERR_ALIGN = -1, -2, -3, -4
+ESPO_ERR_CAPACITY, ESPO_ERR_CUDA, ESPO_ERR_BAD_PARAM = -5, -6, -7
+ESPO_F32, ESPO_BF16 = 0, 1
+ESPO_SAMPLER_FLAT, ESPO_SAMPLER_HIER = 0, 1
+ESPO_ROW_ACTIVE, ESPO_ROW_STOPPED, ESPO_ROW_EOS, ESPO_ROW_TMAX, ESPO_ROW_BAD = 0, 1, 2, 3, 4
+ESPO_DEV_BAD_ROW, ESPO_DEV_BAD_SLOT, ESPO_DEV_TIMEOUT, ESPO_DEV_NAN_VALUE, ESPO_DEV_BAD_LENGTHS = 1, 2, 4, 8, 16
+
+
+class EspoError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().espo_strerror(code).decode()
+        if code == ESPO_ERR_CUDA:
+            msg += f" [cudaError {lib().espo_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+class espo_params(C.Structure):
+    """Mirror of the C struct: parameters frozen for a rollout batch (Eq. 8-10, Algorithm 1)."""
+    _fields_ = [("temperature", C.c_float), ("mu_g", C.c_float), ("sigma2_g", C.c_float),
+                ("delta", C.c_float), ("clip_c", C.c_float), ("alpha_s", C.c_float),
+                ("beta", C.c_float), ("eps", C.c_float), ("warmup_complete", C.c_int32),
+                ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32)]
+
+
+def make_params(temperature=1.0, mu_g=0.0, sigma2_g=1.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0,
+                eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=ESPO_SAMPLER_HIER) -> espo_params:
+    """Defaults follow the paper's hyper-parameter table (alpha_s 0.9, beta 7.0, eps 0.2, T_max 8192)."""
+    return espo_params(temperature, mu_g, sigma2_g, delta, clip_c, alpha_s, beta, eps, warmup_complete, t_max,
+                       eos_token, sampler)
+
+
+_lib = None
+
+
+def lib():
+    """Load ``libespo.so`` (built in-tree).  Raises if it is not there: nothing else can do the work."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build the CUDA library first (python -m paper_2605_29860_b200.build); "
+                "this package has no other implementation to fall back to")
+        L = C.CDLL(path)
+        vp, i32, i64, u64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_float
+        L.espo_init_state.argtypes = [C.POINTER(vp), i32, i32, u64, u64, vp]
+        L.espo_reset_state.argtypes = [vp, u64, vp]
+        L.espo_free_state.argtypes = [vp]
+        L.espo_free_state.restype = None
+        L.espo_set_launch_config.argtypes = [vp, i32, i32]
+        L.espo_step.argtypes = [vp, i32, i64, vp, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp, vp]
+        L.espo_state_view.argtypes = [vp] + [C.POINTER(vp)] * 9
+        L.espo_compact_active.argtypes = [vp, vp, vp, vp]
+        L.espo_state_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        L.espo_advantages.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp]
+        L.espo_advantages_reserve.argtypes = [i32, i64]
+        L.espo_advantages_status.argtypes = [C.POINTER(C.c_uint32), vp]
+        L.espo_strerror.argtypes = [C.c_int]
+        L.espo_strerror.restype = C.c_char_p
+        L.espo_last_cuda_error.argtypes = []
+        for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_state_view",
+                  "espo_compact_active", "espo_state_status", "espo_advantages", "espo_advantages_reserve",
+                  "espo_advantages_status", "espo_last_cuda_error"):
+            getattr(L, n).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != ESPO_OK:
+        raise EspoError(code, where)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev_ptr(t: Optional[torch.Tensor], name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    return t.data_ptr()
+
+
+def _dtype_code(t: torch.Tensor, name: str) -> int:
+    if t.dtype == torch.float32:
+        return ESPO_F32
+    if t.dtype == torch.bfloat16:
+        return ESPO_BF16
+    raise ValueError(f"{name} must be float32 or bfloat16, got {t.dtype}")
+
+
+class EspoState:
+    """Owner of an ``espo_state*``; frees it when collected."""
+
+    def __init__(self, handle: int, capacity: int, V: int, device: torch.device):
+        self.handle = C.c_void_p(handle)
+        self.capacity = capacity
+        self.V = V
+        self.device = device
+
+    def close(self) -> None:
+        if self.handle:
+            lib().espo_free_state(self.handle)
+            self.handle = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def espo_init_state(capacity: int, V: int, seed: int, batch_id: int = 0, stream=None) -> EspoState:
+    if not torch.cuda.is_available():
+        raise RuntimeError("espo_init_state needs a CUDA device; there is no CPU implementation")
+    h = C.c_void_p()
+    _check(lib().espo_init_state(C.byref(h), capacity, V, seed, batch_id, _stream(stream)), "espo_init_state")
+    return EspoState(h.value, capacity, V, torch.device("cuda", torch.cuda.current_device()))
+
+
+def espo_reset_state(state: EspoState, batch_id: int, stream=None) -> None:
+    _check(lib().espo_reset_state(state.handle, batch_id, _stream(stream)), "espo_reset_state")
+
+
+def espo_free_state(state: EspoState) -> None:
+    state.close()
+
+
+def espo_set_launch_config(state: EspoState, stages: int = 0, ctas_per_sm: int = 0) -> None:
+    _check(lib().espo_set_launch_config(state.handle, stages, ctas_per_sm), "espo_set_launch_config")
+
+
+def espo_step(logits: torch.Tensor, values: torch.Tensor, state: EspoState, params: espo_params,
+              tokens_out: torch.Tensor, stop_out: torch.Tensor, row_ids: Optional[torch.Tensor] = None,
+              n_rows: Optional[int] = None, stream=None) -> None:
+    """One decode step (Algorithm 1 loop body) for ``logits`` [n_rows, V]; see ``espo.h``."""
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [n_rows, V] with unit stride along V")
+    n = logits.shape[0] if n_rows is None else n_rows
+    if logits.shape[1] != state.V:
+        raise ValueError(f"logits have V={logits.shape[1]}, state was created for V={state.V}")
+    if tokens_out.dtype != torch.int32 or stop_out.dtype != torch.uint8:
+        raise ValueError("tokens_out must be int32 and stop_out uint8")
+    if row_ids is not None and row_ids.dtype != torch.int32:
+        raise ValueError("row_ids must be int32")
+    if not values.is_contiguous() or not tokens_out.is_contiguous() or not stop_out.is_contiguous():
+        raise ValueError("values, tokens_out and stop_out must be contiguous")
+    if min(values.numel(), tokens_out.numel(), stop_out.numel()) < n or (row_ids is not None and row_ids.numel() < n):
+        raise ValueError("an argument is shorter than n_rows")
+    _check(lib().espo_step(_dev_ptr(logits, "logits"), _dtype_code(logits, "logits"), logits.stride(0),
+                           _dev_ptr(values, "values"), _dtype_code(values, "values"),
+                           _dev_ptr(row_ids, "row_ids"), n, state.handle, C.byref(params),
+                           _dev_ptr(tokens_out, "tokens_out"), _dev_ptr(stop_out, "stop_out"), _stream(stream)),
+           "espo_step")
+
+
+class _DevArray:
+    """Minimal __cuda_array_interface__ carrier so torch can view library-owned device memory."""
+
+    def __init__(self, ptr: int, n: int, typestr: str):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (ptr, False), "version": 2}
+
+
+def espo_state_view(state: EspoState) -> dict:
+    """Torch views (treat as read-only) of the per-slot arrays: z, g, g_tilde, logp, t, status, t_stop, sum_g, sum_g2."""
+    ptrs = [C.c_void_p() for _ in range(9)]
+    _check(lib().espo_state_view(state.handle, *[C.byref(p) for p in ptrs]), "espo_state_view")
+    names = ["z", "g", "g_tilde", "logp", "t", "status", "t_stop", "sum_g", "sum_g2"]
+    types = ["<f4", "<f4", "<f4", "<f4", "<i4", "|u1", "<i4", "<f8", "<f8"]
+    with torch.cuda.device(state.device):
+        return {n: torch.as_tensor(_DevArray(p.value, state.capacity, ty), device=state.device)
+                for n, p, ty in zip(names, ptrs, types)}
+
+
+def espo_compact_active(state: EspoState, row_ids_out: torch.Tensor, n_active_out: torch.Tensor, stream=None) -> None:
+    if row_ids_out.dtype != torch.int32 or n_active_out.dtype != torch.int32:
+        raise ValueError("row_ids_out and n_active_out must be int32")
+    if row_ids_out.numel() < state.capacity or n_active_out.numel() < 1:
+        raise ValueError("row_ids_out must hold capacity entries and n_active_out one")
+    _check(lib().espo_compact_active(state.handle, _dev_ptr(row_ids_out, "row_ids_out"),
+                                     _dev_ptr(n_active_out, "n_active_out"), _stream(stream)), "espo_compact_active")
+
+
+def espo_state_status(state: EspoState, stream=None) -> int:
+    out = C.c_uint32(0)
+    _check(lib().espo_state_status(state.handle, C.byref(out), _stream(stream)), "espo_state_status")
+    return out.value
+
+
+def espo_advantages(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.Tensor, stopped: torch.Tensor,
+                    gamma: float, lam: float, r_fail: float, adv_out: torch.Tensor,
+                    total_tokens: Optional[int] = None, stream=None) -> None:
+    """TD + GAE over packed ragged trajectories with the failure transition (Eq. 3-4, 12); see ``espo.h``."""
+    for t, n, dt in ((rewards, "rewards", torch.float32), (values, "values", torch.float32),
+                     (adv_out, "adv_out", torch.float32), (lengths, "lengths", torch.int32),
+                     (stopped, "stopped", torch.uint8)):
+        if t.dtype != dt or not t.is_contiguous():
+            raise ValueError(f"{n} must be a contiguous {dt} tensor")
+    total = rewards.numel() if total_tokens is None else total_tokens
+    if values.numel() < total or adv_out.numel() < total or rewards.numel() < total:
+        raise ValueError("rewards, values and adv_out must hold total_tokens entries")
+    if stopped.numel() < lengths.numel():
+        raise ValueError("stopped is shorter than lengths")
+    _check(lib().espo_advantages(_dev_ptr(rewards, "rewards"), _dev_ptr(values, "values"),
+                                 _dev_ptr(lengths, "lengths"), _dev_ptr(stopped, "stopped"), lengths.numel(), total,
+                                 gamma, lam, r_fail, _dev_ptr(adv_out, "adv_out"), _stream(stream)),
+           "espo_advantages")
+
+
+def espo_advantages_reserve(max_B: int, max_tokens: int) -> None:
+    _check(lib().espo_advantages_reserve(max_B, max_tokens), "espo_advantages_reserve")
+
+
+def espo_advantages_status(stream=None) -> int:
+    out = C.c_uint32(0)
+    _check(lib().espo_advantages_status(C.byref(out), _stream(stream)), "espo_advantages_status")
+    return out.value

@@ -1,0 +1,158 @@
+// Device-side building blocks shared by the ESPO kernels: mbarrier / bulk-copy PTX
+// wrappers with bounded waits, Philox4x32-10, warp reductions.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace espo {
+
+constexpr int kBlockIds = 1024;  // ids per sampling block (level 2 of the hierarchical sampler)
+constexpr int kSubIds = 32;      // ids per sub-block (level 1)
+constexpr unsigned kFullMask = 0xffffffffu;
+
+// Iteration caps of the in-kernel waits.  A wait that runs out records ESPO_DEV_TIMEOUT and
+// the kernel winds down instead of spinning forever.
+constexpr uint32_t kMbarSpinLimit = 1u << 22;   // try_wait calls (each may suspend in hardware)
+constexpr uint32_t kPollSpinLimit = 1u << 22;   // polls with a short sleep in between
+
+// ---------------------------------------------------------------- shared-memory barriers
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_init_fence() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+               : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Wait for the phase with the given parity, giving up after kMbarSpinLimit tries or as soon
+// as another warp of the CTA has raised `*abort_flag`.  Returns false when it gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kMbarSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u && *abort_flag) return false;
+  }
+  return false;
+}
+
+// Bulk asynchronous copy global -> shared (TMA, no tensor map, no multicast).  Both addresses
+// 16-byte aligned, bytes a multiple of 16.  Completion is signalled on `bar` as transaction bytes.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_addr(dst_smem)),
+      "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+      : "memory");
+}
+
+// ---------------------------------------------------------------- Philox4x32-10
+
+// Counter-based generator of Salmon et al. (SC'11): ten rounds, each two 32x32->64 multiplies
+// and a key-dependent xor; the key advances by the Weyl constants between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                               uint32_t k1) {
+  constexpr uint32_t MA = 0xD2511F53u, MB = 0xCD9E8D57u, WA = 0x9E3779B9u, WB = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t ha = __umulhi(MA, c0), la = MA * c0;
+    const uint32_t hb = __umulhi(MB, c2), lb = MB * c2;
+    const uint32_t n0 = hb ^ c1 ^ k0;
+    const uint32_t n2 = ha ^ c3 ^ k1;
+    c0 = n0; c1 = lb; c2 = n2; c3 = la;
+    k0 += WA; k1 += WB;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint32_t pick_word(const uint4& w, uint32_t i) {
+  return i == 0 ? w.x : (i == 1 ? w.y : (i == 2 ? w.z : w.w));
+}
+
+// 23 random bits k -> u = (2k+1)/2^24 in (0,1), exact in float32; G = -log(-log u), full-precision logs.
+__device__ __forceinline__ float gumbel_from_word(uint32_t word) {
+  const float u = __uint2float_rn(2u * (word >> 9) + 1u) * 5.9604644775390625e-08f;
+  return -logf(-logf(u));
+}
+
+// Which Philox stream a draw belongs to: (step, slot, batch|level) are counter words 1..3.
+struct DrawStream {
+  uint32_t k0, k1;     // seed halves
+  uint32_t step, slot;
+  uint32_t batch_bits; // batch_id << 2
+};
+
+__device__ __forceinline__ float gumbel_at(const DrawStream& ds, uint32_t level, uint32_t index) {
+  const uint4 w = philox4x32_10(index >> 2, ds.step, ds.slot, ds.batch_bits | level, ds.k0, ds.k1);
+  return gumbel_from_word(pick_word(w, index & 3u));
+}
+
+// ---------------------------------------------------------------- warp reductions
+
+__device__ __forceinline__ float warp_max(float v) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+  return r;
+}
+
+// Butterfly sum: every lane ends with the same bits, independent of anything but the inputs.
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+  return v;
+}
+
+// Argmax of (score, index) over the warp; the lower index wins equal scores.  Lanes with
+// nothing to offer pass index < 0.  Every lane gets the result.
+__device__ __forceinline__ void warp_argmax(float& score, int& index) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float s2 = __shfl_xor_sync(kFullMask, score, o);
+    const int i2 = __shfl_xor_sync(kFullMask, index, o);
+    const bool take = (i2 >= 0) && (index < 0 || s2 > score || (s2 == score && i2 < index));
+    if (take) { score = s2; index = i2; }
+  }
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+  uint32_t c;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(c) : "r"(a), "r"(b));
+  return c;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+}  // namespace espo

@@ -1,0 +1,85 @@
+"""GPU parity of espo_advantages against the CPU oracle, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_29860_b200 as espo
+from paper_2605_29860_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(rewards, values, lengths, stopped, gamma, lam, r_fail):
+    total = rewards.numel()
+    adv = torch.full((max(total, 1),), float("nan"), device="cuda")
+    espo.espo_advantages(rewards, values, lengths, stopped, gamma, lam, r_fail, adv, total_tokens=total)
+    torch.cuda.synchronize()
+    assert espo.espo_advantages_status() == 0
+    ref = oracle.advantages(rewards.cpu().numpy(), values.cpu().numpy(), lengths.cpu().numpy(),
+                            stopped.cpu().numpy(), gamma, lam, r_fail)
+    got = adv[:total].cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref)
+    tol = 1e-5 + 1e-4 * np.abs(ref)
+    bad = np.nonzero(~(err <= tol))[0]
+    assert bad.size == 0, f"{bad.size} of {total} advantages off; first at {bad[:5]}: gpu {got[bad[:5]]} ref {ref[bad[:5]]}"
+    return float(err.max()) if total else 0.0
+
+
+@pytest.mark.parametrize("lam", [0.95, 1.0])
+def test_config5_ragged_batch(lam):
+    # B=1024, lengths U[256,16384], 35% stopped (terminal r_fail=-1), others Bernoulli terminal reward
+    r, v, L, s = synth.ragged_trajectories(1024, seed=0)
+    assert r.numel() > 8_000_000
+    _check(r, v, L, s, 1.0, lam, -1.0)
+
+
+@pytest.mark.parametrize("gamma,lam", [(0.99, 0.9), (1.0, 0.0), (0.0, 0.5)])
+def test_discount_variants(gamma, lam):
+    r, v, L, s = synth.ragged_trajectories(200, len_lo=1, len_hi=5000, seed=1)
+    _check(r, v, L, s, gamma, lam, -1.0)
+
+
+@pytest.mark.parametrize("lengths", [[1], [2048], [2047], [2049], [4096, 4096], [1] * 5000, [0, 3, 0, 0, 2050, 0],
+                                     [70000], [2048, 1, 2047, 4097, 5], [3, 2045, 2048, 2048, 1]])
+def test_edge_lengths(lengths):
+    g = torch.Generator("cuda").manual_seed(len(lengths) + sum(lengths))
+    L = torch.tensor(lengths, dtype=torch.int32, device="cuda")
+    total = int(sum(lengths))
+    r = torch.randn(total, device="cuda", generator=g) * 0.5
+    v = torch.randn(total, device="cuda", generator=g) * 0.5
+    s = (torch.rand(len(lengths), device="cuda", generator=g) < 0.5).to(torch.uint8)
+    _check(r, v, L, s, 1.0, 1.0, -1.0)
+    _check(r, v, L, s, 0.98, 0.97, -0.5)
+
+
+def test_replace_not_add_and_repeat_calls_bit_identical():
+    r, v, L, s = synth.ragged_trajectories(64, len_lo=1, len_hi=9000, seed=3)
+    last = (torch.cumsum(L.long(), 0) - 1)
+    r[last] = 0.7                       # a stopped trajectory's stored last reward must be replaced
+    _check(r, v, L, s, 1.0, 0.95, -1.0)
+    outs = []
+    for _ in range(3):
+        adv = torch.empty_like(r)
+        espo.espo_advantages(r, v, L, s, 1.0, 0.95, -1.0, adv)
+        outs.append(adv.clone())
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+
+
+def test_inconsistent_lengths_are_reported_not_trapped():
+    r, v, L, s = synth.ragged_trajectories(16, len_lo=10, len_hi=100, seed=4)
+    adv = torch.empty_like(r)
+    espo.espo_advantages(r, v, L, s, 1.0, 0.95, -1.0, adv, total_tokens=r.numel() - 3)
+    torch.cuda.synchronize()
+    assert espo.espo_advantages_status() & espo.ESPO_DEV_BAD_LENGTHS
+    assert espo.espo_advantages_status() == 0            # reading clears it
+    with pytest.raises(espo.EspoError) as e:
+        espo.espo_advantages(r[1:], v[1:], L, s, 1.0, 0.95, -1.0, adv[1:], total_tokens=8)
+    assert e.value.code == espo.ESPO_ERR_ALIGN
+
+
+def test_reserve_then_smaller_calls():
+    espo.espo_advantages_reserve(2048, 20_000_000)
+    for seed in (5, 6):
+        r, v, L, s = synth.ragged_trajectories(300, len_lo=1, len_hi=3000, seed=seed)
+        _check(r, v, L, s, 1.0, 0.95, -1.0)
