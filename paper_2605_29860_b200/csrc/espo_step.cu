@@ -297,6 +297,16 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
   }
   S = warp_sum(S);
   warp_argmax(best, best_i);
+  if (best_i < 0) {   // no block offered a candidate: treat like an unusable row rather than index with -1
+    if (lane == 0) {
+      atomicOr(a.dev_status, ESPO_DEV_BAD_ROW);
+      a.status[slot] = ESPO_ROW_BAD;
+      a.tokens_out[row] = 0;
+      a.stop_out[row] = 0;
+      a.ticket[row] = 0;
+    }
+    return;
+  }
 
   int token;
   float l_tok;
@@ -365,7 +375,7 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
         if (l > NINF) { sc0 = (l - M) * a.inv_temp + gumbel_at(ds, 0u, (uint32_t)id); cand = id; }
       }
       warp_argmax(sc0, cand);
-      token = cand;
+      token = max(cand, sub_pick * kSubIds);   // cand < 0 cannot happen for a sub-block with a finite id
       l_tok = __shfl_sync(kFullMask, l, token & 31);
     }
     (void)sub_pick;
