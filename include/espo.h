@@ -190,6 +190,37 @@ int espo_advantages_reserve(int32_t max_B, int64_t max_tokens);
  * of the current device to *host_out and clear it.  Synchronises `stream`. */
 int espo_advantages_status(uint32_t* host_out, void* stream);
 
+/* Limits of espo_advantages_noalloc. */
+#define ESPO_NOALLOC_MAX_B       4096          /* trajectories per call                          */
+#define ESPO_NOALLOC_MAX_TOKENS  16777216      /* sum(lengths) per call (2^24)                   */
+
+/* espo_advantages for callers that must not allocate device memory.  (The paper has no
+ * counterpart of this entry point; it computes exactly what espo_advantages computes.)
+ *
+ * Who needs it: a rollout worker whose serving engine claimed all free device memory for its
+ * own pools at start-up, so that a cudaMalloc issued by a library fails; and a training loop
+ * that cannot afford the device-wide synchronisation that cudaMalloc/cudaFree imply.  This call
+ * never calls cudaMalloc, cudaFree or any other allocating routine: its scratch is a fixed
+ * array of about 0.3 MB that is part of the library image, so every device that loads the
+ * library holds that array until the process exits.
+ *
+ * Arguments are those of espo_advantages, plus
+ *   status_out   device uint32 [1] or NULL: ESPO_DEV_TIMEOUT / ESPO_DEV_BAD_LENGTHS bits are
+ *                OR-ed into it (the caller clears it); with NULL they go to a word inside the
+ *                scratch that cannot be read back.
+ * Limits: B <= ESPO_NOALLOC_MAX_B and total_tokens <= ESPO_NOALLOC_MAX_TOKENS, otherwise
+ * ESPO_ERR_CAPACITY and nothing is launched.
+ * The first call on each device looks up the scratch array's device address (with that device
+ * current) and remembers it; make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents; the
+ * call itself clears the part that has to start at zero.  Two calls that overlap on the
+ * device (different streams, no dependency) race on it: serialise them.
+ * Errors: BAD_SHAPE, CAPACITY, NULL, ALIGN (16-byte arrays), BAD_PARAM, CUDA. */
+int espo_advantages_noalloc(const float* rewards, const float* values, const int32_t* lengths,
+                            const uint8_t* stopped, int32_t B, int64_t total_tokens,
+                            float gamma, float lambda, float r_fail, float* adv_out,
+                            uint32_t* status_out, void* stream);
+
 /* Text for a return code; never NULL. */
 const char* espo_strerror(int code);
 

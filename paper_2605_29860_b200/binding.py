@@ -71,6 +71,7 @@ def lib():
         L.espo_compact_active.argtypes = [vp, vp, vp, vp]
         L.espo_state_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.espo_advantages.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp]
+        L.espo_advantages_noalloc.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp]
         L.espo_advantages_reserve.argtypes = [i32, i64]
         L.espo_advantages_status.argtypes = [C.POINTER(C.c_uint32), vp]
         L.espo_strerror.argtypes = [C.c_int]
@@ -78,7 +79,7 @@ def lib():
         L.espo_last_cuda_error.argtypes = []
         for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_state_view",
                   "espo_compact_active", "espo_state_status", "espo_advantages", "espo_advantages_reserve",
-                  "espo_advantages_status", "espo_last_cuda_error"):
+                  "espo_advantages_status", "espo_advantages_noalloc", "espo_last_cuda_error"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -227,6 +228,36 @@ def espo_advantages(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.
                                  _dev_ptr(lengths, "lengths"), _dev_ptr(stopped, "stopped"), lengths.numel(), total,
                                  gamma, lam, r_fail, _dev_ptr(adv_out, "adv_out"), _stream(stream)),
            "espo_advantages")
+
+
+ESPO_NOALLOC_MAX_B, ESPO_NOALLOC_MAX_TOKENS = 4096, 1 << 24
+
+
+def espo_advantages_noalloc(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.Tensor, stopped: torch.Tensor,
+                            gamma: float, lam: float, r_fail: float, adv_out: torch.Tensor,
+                            status_out: Optional[torch.Tensor] = None, total_tokens: Optional[int] = None,
+                            stream=None) -> None:
+    """``espo_advantages`` for processes that cannot allocate device memory (the engine owns it all, or a
+    cudaMalloc's device-wide synchronisation is not acceptable): the library's scratch is a fixed array inside
+    the library image.  At most ESPO_NOALLOC_MAX_B trajectories and ESPO_NOALLOC_MAX_TOKENS tokens per call.
+    ``status_out`` (int32/uint32 CUDA tensor of one element, or None) receives the ESPO_DEV_* bits."""
+    for t, n, dt in ((rewards, "rewards", torch.float32), (values, "values", torch.float32),
+                     (adv_out, "adv_out", torch.float32), (lengths, "lengths", torch.int32),
+                     (stopped, "stopped", torch.uint8)):
+        if t.dtype != dt or not t.is_contiguous():
+            raise ValueError(f"{n} must be a contiguous {dt} tensor")
+    total = rewards.numel() if total_tokens is None else total_tokens
+    if values.numel() < total or adv_out.numel() < total or rewards.numel() < total:
+        raise ValueError("rewards, values and adv_out must hold total_tokens entries")
+    if stopped.numel() < lengths.numel():
+        raise ValueError("stopped is shorter than lengths")
+    if status_out is not None and (status_out.element_size() != 4 or status_out.numel() < 1):
+        raise ValueError("status_out must hold one 32-bit word")
+    _check(lib().espo_advantages_noalloc(_dev_ptr(rewards, "rewards"), _dev_ptr(values, "values"),
+                                         _dev_ptr(lengths, "lengths"), _dev_ptr(stopped, "stopped"),
+                                         lengths.numel(), total, gamma, lam, r_fail, _dev_ptr(adv_out, "adv_out"),
+                                         _dev_ptr(status_out, "status_out"), _stream(stream)),
+           "espo_advantages_noalloc")
 
 
 def espo_advantages_reserve(max_B: int, max_tokens: int) -> None:

@@ -332,9 +332,88 @@ static int ensure_pool(int dev, int B, long long nchunks, AdvPool** out) {
   return ESPO_OK;
 }
 
+// ---------------------------------------------------------------------------------------
+// Fixed scratch for espo_advantages_noalloc: the same workspace layout as AdvPool's arena,
+// carved out of an array that is part of the loaded module, sized for kNoAllocMaxB
+// trajectories and kNoAllocMaxChunks chunks.  Zero-filled when the module is loaded.
+// ---------------------------------------------------------------------------------------
+constexpr int kNoAllocMaxB = ESPO_NOALLOC_MAX_B;
+constexpr long long kNoAllocMaxChunks = (ESPO_NOALLOC_MAX_TOKENS + kAdvChunk - 1) / kAdvChunk;
+constexpr size_t kNaOffOffsets = 0;
+constexpr size_t kNaOffChunkFirst = kNaOffOffsets + ((8 * ((size_t)kNoAllocMaxB + 1) + 255) / 256) * 256;
+constexpr size_t kNaOffFlag = kNaOffChunkFirst + 4 * (size_t)kNoAllocMaxChunks;
+constexpr size_t kNaOffAgg = kNaOffFlag + 4 * (size_t)kNoAllocMaxChunks;
+constexpr size_t kNaOffFin = kNaOffAgg + 16 * (size_t)kNoAllocMaxChunks;
+constexpr size_t kNaOffCounters = kNaOffFin + 8 * (size_t)kNoAllocMaxChunks;
+constexpr size_t kNaOffStatus = kNaOffCounters + 256;
+constexpr size_t kNoAllocBytes = kNaOffStatus + 256;
+static_assert(kNoAllocMaxChunks % 64 == 0, "keeps every sub-array 256-byte aligned");
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+struct NoAllocSlot {
+  unsigned char* base = nullptr;   // device address of g_noalloc_scratch on this device
+  unsigned epoch = 0;
+};
+static NoAllocSlot g_noalloc[kMaxDevices];
+
 }  // namespace espo
 
 extern "C" {
+
+int espo_advantages_noalloc(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
+                            int32_t B, int64_t total_tokens, float gamma, float lambda, float r_fail, float* adv_out,
+                            uint32_t* status_out, void* stream) {
+  using namespace espo;
+  if (B < 0 || total_tokens < 0) return ESPO_ERR_BAD_SHAPE;
+  if (B > kNoAllocMaxB || total_tokens > (int64_t)ESPO_NOALLOC_MAX_TOKENS) return ESPO_ERR_CAPACITY;
+  if (B == 0 || total_tokens == 0) return ESPO_OK;
+  if (!rewards || !values || !lengths || !stopped || !adv_out) return ESPO_ERR_NULL;
+  if (((uintptr_t)rewards % 16) || ((uintptr_t)values % 16) || ((uintptr_t)adv_out % 16) || ((uintptr_t)lengths % 4) ||
+      ((uintptr_t)status_out % 4))
+    return ESPO_ERR_ALIGN;
+  if (gamma != gamma || lambda != lambda || r_fail != r_fail) return ESPO_ERR_BAD_PARAM;
+  const long long nchunks = (total_tokens + kAdvChunk - 1) / kAdvChunk;
+  int dev;
+  ESPO_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return ESPO_ERR_CAPACITY;
+  std::lock_guard<std::mutex> lk(g_pool_mu);
+  NoAllocSlot& slot = g_noalloc[dev];
+  if (!slot.base) {
+    // In host code the array's name is only a handle; the kernels need its address on this device.
+    void* p = nullptr;
+    ESPO_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    slot.base = static_cast<unsigned char*>(p);
+    slot.epoch = 0;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  unsigned char* b = slot.base;
+  if (++slot.epoch >= (1u << 30)) {   // the descriptors' flags carry the epoch; start over before it wraps
+    ESPO_CUDA_TRY(cudaMemsetAsync(b + kNaOffFlag, 0, 4 * (size_t)kNoAllocMaxChunks, s));
+    slot.epoch = 1;
+  }
+  // The array keeps whatever the previous call left: the chunk tickets must start at zero even if
+  // that call was cut short, and the built-in status word is only ever OR-ed into.
+  ESPO_CUDA_TRY(cudaMemsetAsync(b + kNaOffCounters, 0, 8, s));
+  AdvArgs a;
+  a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out;
+  a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
+  a.gamma = (double)gamma; a.gl = (double)gamma * (double)lambda;
+  a.r_fail = r_fail;
+  a.epoch4 = slot.epoch << 2;
+  a.ws.offsets = (long long*)(b + kNaOffOffsets);
+  a.ws.chunk_first = (int*)(b + kNaOffChunkFirst);
+  a.ws.flag = (unsigned*)(b + kNaOffFlag);
+  a.ws.agg = (double2*)(b + kNaOffAgg);
+  a.ws.fin = (double*)(b + kNaOffFin);
+  a.ws.counters = (unsigned*)(b + kNaOffCounters);
+  a.ws.status = status_out ? status_out : (unsigned*)(b + kNaOffStatus);
+  espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
+  ESPO_CUDA_TRY(cudaGetLastError());
+  espo_adv_scan_kernel<<<(unsigned)nchunks, kAdvThreads, 0, s>>>(a);
+  ESPO_CUDA_TRY(cudaGetLastError());
+  return ESPO_OK;
+}
 
 int espo_advantages_reserve(int32_t max_B, int64_t max_tokens) {
   using namespace espo;
