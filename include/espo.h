@@ -148,10 +148,12 @@ int espo_state_view(espo_state* st, const float** z, const float** g, const floa
                     const float** logp, const int32_t** t, const uint8_t** status,
                     const int32_t** t_stop, const double** sum_g, const double** sum_g2);
 
-/* Expert knob: override the step kernel's launch shape for this state.  stages = number of
- * shared-memory ring stages per CTA, ctas_per_sm = resident CTAs per SM; 0 keeps the
- * library default for either.  Results never depend on it.  Errors: NULL, BAD_PARAM. */
-int espo_set_launch_config(espo_state* st, int32_t stages, int32_t ctas_per_sm);
+/* Expert knob: override the step kernel's launch shape for this state.  consumer_warps =
+ * streaming warps per CTA (1..31), stages = blocks of 1024 ids each warp keeps in flight,
+ * ctas_per_sm = resident CTAs per SM; 0 keeps the library default for any of them, and the
+ * library shrinks what does not fit in shared memory.  Results never depend on it.
+ * Errors: NULL, BAD_PARAM. */
+int espo_set_launch_config(espo_state* st, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm);
 
 /* Stable compaction of the active set: writes the slots whose status is ESPO_ROW_ACTIVE, in
  * increasing order, to row_ids_out (device int32 [capacity]) and their number to

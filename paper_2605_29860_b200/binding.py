@@ -65,7 +65,7 @@ def lib():
         L.espo_reset_state.argtypes = [vp, u64, vp]
         L.espo_free_state.argtypes = [vp]
         L.espo_free_state.restype = None
-        L.espo_set_launch_config.argtypes = [vp, i32, i32]
+        L.espo_set_launch_config.argtypes = [vp, i32, i32, i32]
         L.espo_step.argtypes = [vp, i32, i64, vp, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp, vp]
         L.espo_state_view.argtypes = [vp] + [C.POINTER(vp)] * 9
         L.espo_compact_active.argtypes = [vp, vp, vp, vp]
@@ -149,8 +149,8 @@ def espo_free_state(state: EspoState) -> None:
     state.close()
 
 
-def espo_set_launch_config(state: EspoState, stages: int = 0, ctas_per_sm: int = 0) -> None:
-    _check(lib().espo_set_launch_config(state.handle, stages, ctas_per_sm), "espo_set_launch_config")
+def espo_set_launch_config(state: EspoState, consumer_warps: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
+    _check(lib().espo_set_launch_config(state.handle, consumer_warps, stages, ctas_per_sm), "espo_set_launch_config")
 
 
 def espo_step(logits: torch.Tensor, values: torch.Tensor, state: EspoState, params: espo_params,

@@ -53,13 +53,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Wait for the phase with the given parity, giving up after kMbarSpinLimit tries or as soon
-// as another warp of the CTA has raised `*abort_flag`.  Returns false when it gave up.
+// as another warp of the CTA has raised `*abort_flag` (may be null).  Returns false when it gave up.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kMbarSpinLimit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && *abort_flag) return false;
+    if ((it & 255u) == 255u && abort_flag && *abort_flag) return false;
   }
   return false;
+}
+
+// Orders this thread's earlier generic-proxy accesses to shared memory before later
+// asynchronous-proxy ones (a bulk copy that overwrites a stage the warp has just read).
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
 // Bulk asynchronous copy global -> shared (TMA, no tensor map, no multicast).  Both addresses

@@ -6,19 +6,25 @@
 // (Eq. 10) and the per-trajectory bookkeeping.
 //
 // Shape of the kernel
-//   * The [n_rows, V] logits are cut into tiles of kConsumerWarps blocks of 1024 ids.  A
-//     persistent grid (a multiple of the SM count) splits the tile sequence into equal
-//     contiguous ranges, so every SM streams the same number of bytes whatever n_rows is.
-//   * Inside a CTA one producer thread moves tiles from HBM into a ring of shared-memory
-//     stages with bulk asynchronous copies (TMA without a tensor map) that complete on
-//     mbarriers; eight consumer warps each reduce one 1024-id block of the tile to
-//     (max logit, sum of exp) -- plus, for the flat sampler, the block's best perturbed
-//     score -- and write that record to a small per-row table in global memory.
-//   * A row may be spread over several CTAs.  Each consumer warp counts the blocks it has
-//     contributed to a row and adds them to the row's ticket; whoever completes the ticket
-//     hands the row to its CTA's finalizer warp, which merges the block records in a fixed
-//     order (so results do not depend on the grid), draws the token, applies Eq. 5, 8, 9, 10
-//     and writes the outputs and the trajectory state.  The streaming warps never wait for it.
+//   * The [n_rows, V] logits are a sequence of n_rows * ceil(V/1024) blocks of 1024 ids.  A
+//     persistent grid (a multiple of the SM count) splits that sequence into equal contiguous
+//     ranges, so every SM streams the same number of bytes whatever n_rows is.
+//   * Inside a CTA every streaming warp owns a private ring of shared-memory stages, one block
+//     each.  Its lane 0 fetches the warp's next blocks with bulk asynchronous copies (TMA
+//     without a tensor map) that complete on the stage's mbarrier; the warp reduces a block
+//     to (max logit, sum of exp) -- plus, for the flat sampler, the block's best perturbed
+//     score -- writes that record to a per-row table in global memory and refills the stage.
+//     Warps never wait for one another.
+//   * A row may be spread over several CTAs.  The warps of a CTA count the blocks they have
+//     contributed to a row in shared memory; when the CTA's share of the row is complete the
+//     row is posted to a small queue.  The CTA's finalizer warp (and, once they run out of
+//     blocks, the streaming warps) take rows from the queue, add the CTA's share to the
+//     row's ticket in global memory, and whoever completes the ticket merges the block
+//     records in a fixed order (so results do not depend on the grid), draws the token,
+//     applies Eq. 5, 8, 9, 10 and writes the outputs and the trajectory state.
+//   * A CTA walks its range starting with the row it shares with the next CTA, then the row it
+//     shares with the previous one, then its whole rows: shared rows complete early in the
+//     launch instead of all at its end.
 //   * Every wait in the kernel is bounded; a wait that runs out sets ESPO_DEV_TIMEOUT.
 #include <cuda_runtime.h>
 #include <math.h>
@@ -33,11 +39,10 @@
 
 namespace espo {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kStepThreads = (kConsumerWarps + 2) * 32;   // + producer warp + finalizer warp
-constexpr int kProducerWarp = kConsumerWarps;
-constexpr int kFinalizerWarp = kConsumerWarps + 1;
+constexpr int kMaxStepThreads = 1024;
+constexpr int kMaxConsumerWarps = kMaxStepThreads / 32 - 1;   // one more warp is the finalizer
 constexpr int kMaxQueue = 4096;
+constexpr int kRegRecords = 8;    // block records a finalizer lane keeps in registers (covers V <= 262144)
 
 struct StepArgs {
   // inputs
@@ -48,10 +53,9 @@ struct StepArgs {
   const int32_t* row_ids;
   int n_rows, V, capacity;
   // tiling
-  int nblk;             // 1024-id blocks per row
-  int tiles_per_row;
-  long long total_tiles;
-  int stages, tile_bytes, queue_cap;
+  int nblk;                 // 1024-id blocks per row
+  long long total_blocks;   // n_rows * nblk
+  int warps, stages, stage_bytes, queue_cap;
   // trajectory state (indexed by slot)
   float *z, *g, *g_tilde, *logp;
   int32_t *t, *t_stop;
@@ -74,8 +78,8 @@ struct StepArgs {
 };
 
 struct StepCtrl {
-  int fin_tail;     // rows handed to the finalizer so far
-  int done_warps;   // consumer warps that have left their loop
+  int head;         // queue entries claimed so far
+  int posted;       // queue entries posted so far
   int abort_flag;   // a bounded wait ran out somewhere in this CTA
   int pad;
 };
@@ -105,7 +109,7 @@ struct BlockVals<2> {   // bfloat16: 4 vectors of 8 ids per lane
       for (int i = 0; i < kVecs; ++i) {
         const int first = (i * 32 + lane) * kPerVec;
         uint4 q = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-        if (first < nvalid) q = sp[i * 32 + lane];
+        if (first < nvalid) q = sp[i * 32 + lane];   // the stage is a full block long; the excess is masked below
         uint32_t ww[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -123,6 +127,7 @@ struct BlockVals<2> {   // bfloat16: 4 vectors of 8 ids per lane
     return fmaxf(bf16_lo(m), bf16_hi(m));
   }
   __device__ __forceinline__ float val(int j) const { return (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]); }
+  __device__ __forceinline__ float2 pair(int j) const { return make_float2(bf16_lo(w[j]), bf16_hi(w[j])); }
 };
 
 template <>
@@ -143,7 +148,7 @@ struct BlockVals<4> {   // float32: 8 vectors of 4 ids per lane
       for (int i = 0; i < kVecs; ++i) {
         const int first = (i * 32 + lane) * kPerVec;
         float4 q = make_float4(ninf, ninf, ninf, ninf);
-        if (first < nvalid) q = sp[i * 32 + lane];
+        if (first < nvalid) q = sp[i * 32 + lane];   // the stage is a full block long; the excess is masked below
         f[4 * i + 0] = q.x;
         f[4 * i + 1] = (first + 1 < nvalid) ? q.y : ninf;
         f[4 * i + 2] = (first + 2 < nvalid) ? q.z : ninf;
@@ -158,6 +163,7 @@ struct BlockVals<4> {   // float32: 8 vectors of 4 ids per lane
     return m;
   }
   __device__ __forceinline__ float val(int j) const { return f[j]; }
+  __device__ __forceinline__ float2 pair(int j) const { return make_float2(f[2 * j], f[2 * j + 1]); }
 };
 
 // Position inside the block of the j-th value a lane holds.
@@ -174,15 +180,21 @@ __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned c
   bv.load(blk, lane, nvalid);
   const float m_b = warp_max(bv.lane_max());
   const float ref = (m_b == __int_as_float(0xff800000)) ? 0.0f : m_b;   // an all -inf block sums to 0
+  // sum of 2^((x - ref) * k2): two ids per packed fp32 multiply-add and add, one exponential each
+  const float2 k2v = make_float2(a.k2, a.k2);
   const float c0 = -ref * a.k2;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  const float2 c0v = make_float2(c0, c0);
+  float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-  for (int j = 0; j < 32; ++j) acc[(ES == 2 ? (j >> 1) : j) & 3] += ex2_approx(fmaf(bv.val(j), a.k2, c0));
-  const float s_b = warp_sum((acc[0] + acc[1]) + (acc[2] + acc[3]));
+  for (int j = 0; j < 16; ++j) {
+    const float2 t = __ffma2_rn(bv.pair(j), k2v, c0v);
+    const float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
+    if (j & 1) acc1 = __fadd2_rn(acc1, e); else acc0 = __fadd2_rn(acc0, e);
+  }
+  const float s_b = warp_sum((acc0.x + acc0.y) + (acc1.x + acc1.y));
 
   if (SAMPLER == ESPO_SAMPLER_FLAT) {
     // one Philox block serves 4 consecutive ids; a lane's vector starts at a multiple of 4
-    constexpr int P = BlockVals<ES>::kPerVec;
     float best = __int_as_float(0xff800000);
     int best_id = -1;
 #pragma unroll
@@ -196,7 +208,6 @@ __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned c
         if (sc > best) { best = sc; best_id = first + e; }
       }
     }
-    (void)P;
     warp_argmax(best, best_id);
     if (lane == 0)
       a.records[(size_t)row * a.nblk + block] = make_float4(m_b, s_b, best, __int_as_float(best_id));
@@ -215,73 +226,84 @@ __device__ __forceinline__ float load_logit(const unsigned char* row_base, int i
   return __ldg(reinterpret_cast<const float*>(row_base) + id);
 }
 
+__device__ __forceinline__ void mark_row(const StepArgs& a, int row, int slot, int lane, int32_t token, unsigned dev_bit,
+                                         int new_status) {
+  if (lane == 0) {
+    if (dev_bit) atomicOr(a.dev_status, dev_bit);
+    if (new_status >= 0) a.status[slot] = (uint8_t)new_status;
+    a.tokens_out[row] = token;
+    a.stop_out[row] = 0;
+    a.ticket[row] = 0;   // ready for the next launch
+  }
+}
+
 template <int ES, int SAMPLER>
-__device__ void finalize_row(const StepArgs& a, int row, int lane) {
+__device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane) {
   const float NINF = __int_as_float(0xff800000);
-  int slot = a.row_ids ? __ldg(a.row_ids + row) : row;
-  if (slot < 0 || slot >= a.capacity) {
-    if (lane == 0) {
-      atomicOr(a.dev_status, ESPO_DEV_BAD_SLOT);
-      a.tokens_out[row] = -1;
-      a.stop_out[row] = 0;
-      a.ticket[row] = 0;
-    }
-    return;
-  }
-  if (a.status[slot] != ESPO_ROW_ACTIVE) {   // finished trajectories are left untouched
-    if (lane == 0) {
-      a.tokens_out[row] = -1;
-      a.stop_out[row] = 0;
-      a.ticket[row] = 0;
-    }
-    return;
-  }
+  const int slot = a.row_ids ? __ldg(a.row_ids + row) : row;
+  if (slot < 0 || slot >= a.capacity) { mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1); return; }
+  if (a.status[slot] != ESPO_ROW_ACTIVE) { mark_row(a, row, slot, lane, -1, 0u, -1); return; }   // finished: untouched
+
+  // per-trajectory state and the critic value: requested now, used at the very end
   const int t_now = a.t[slot];
+  const float z_prev = a.z[slot];
+  float v;
+  if (a.values_bf16) v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(a.values) + row) << 16);
+  else v = __ldg(reinterpret_cast<const float*>(a.values) + row);
+
   const unsigned char* row_base = a.logits + (size_t)row * a.row_stride_bytes;
   const DrawStream ds{a.key0, a.key1, (uint32_t)t_now, (uint32_t)slot, a.batch_bits};
 
-  // ---- merge the block records: M = max logit, S = sum_b s_b exp((m_b - M)/T) ----
-  float M = NINF;
-  bool poisoned = false;
-  for (int b = lane; b < a.nblk; b += 32) {
-    float m_b, s_b;
+  // ---- the row's block records: lane l owns blocks l, l+32, ...; up to kRegRecords of them stay in registers ----
+  const bool in_regs = a.nblk <= 32 * kRegRecords;
+  float rm[kRegRecords], rs[kRegRecords];
+  float4 rf[SAMPLER == ESPO_SAMPLER_FLAT ? kRegRecords : 1];
+  auto fetch = [&](int b, float& m_b, float& s_b, float& fbest, int& fid) {
     if (SAMPLER == ESPO_SAMPLER_FLAT) {
       const float4 r = __ldcg(a.records + (size_t)row * a.nblk + b);
-      m_b = r.x; s_b = r.y;
+      m_b = r.x; s_b = r.y; fbest = r.z; fid = __float_as_int(r.w);
     } else {
       const float2 r = __ldcg(reinterpret_cast<const float2*>(a.records) + (size_t)row * a.nblk + b);
-      m_b = r.x; s_b = r.y;
+      m_b = r.x; s_b = r.y; fbest = NINF; fid = -1;
     }
-    M = fmaxf(M, m_b);
-    poisoned |= !(s_b >= 0.0f) || isinf(s_b);   // NaN or inf sum: the block held NaN or +inf
+  };
+  float M = NINF;
+  bool poisoned = false;
+  if (in_regs) {
+#pragma unroll
+    for (int i = 0; i < kRegRecords; ++i) {
+      const int b = lane + 32 * i;
+      rm[i] = NINF; rs[i] = 0.f;
+      if (SAMPLER == ESPO_SAMPLER_FLAT) rf[i] = make_float4(0.f, 0.f, NINF, __int_as_float(-1));
+      if (b < a.nblk) {
+        float fb; int fi;
+        fetch(b, rm[i], rs[i], fb, fi);
+        if (SAMPLER == ESPO_SAMPLER_FLAT) rf[i] = make_float4(0.f, 0.f, fb, __int_as_float(fi));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kRegRecords; ++i) {
+      M = fmaxf(M, rm[i]);
+      poisoned |= !(rs[i] >= 0.0f) || isinf(rs[i]);   // NaN or inf sum: the block held NaN or +inf
+    }
+  } else {
+    for (int b = lane; b < a.nblk; b += 32) {
+      float m_b, s_b, fb; int fi;
+      fetch(b, m_b, s_b, fb, fi);
+      M = fmaxf(M, m_b);
+      poisoned |= !(s_b >= 0.0f) || isinf(s_b);
+    }
   }
   M = warp_max(M);
   poisoned = __any_sync(kFullMask, poisoned) || !(M > NINF) || isinf(M);
-  if (poisoned) {
-    if (lane == 0) {
-      atomicOr(a.dev_status, ESPO_DEV_BAD_ROW);
-      a.status[slot] = ESPO_ROW_BAD;
-      a.tokens_out[row] = 0;
-      a.stop_out[row] = 0;
-      a.ticket[row] = 0;
-    }
-    return;
-  }
+  if (poisoned) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD); return; }
 
+  // ---- merge: S = sum_b s_b exp((m_b - M)/T); pick the block (HIER) or the id (FLAT) ----
   float S = 0.f;              // lane-partial, summed below
   float best = NINF;          // best perturbed score among this lane's blocks
-  int best_i = -1;            // HIER: block number; FLAT: token id
-  for (int b = lane; b < a.nblk; b += 32) {
-    float m_b, s_b, flat_best = NINF;
-    int flat_id = -1;
-    if (SAMPLER == ESPO_SAMPLER_FLAT) {
-      const float4 r = __ldcg(a.records + (size_t)row * a.nblk + b);
-      m_b = r.x; s_b = r.y; flat_best = r.z; flat_id = __float_as_int(r.w);
-    } else {
-      const float2 r = __ldcg(reinterpret_cast<const float2*>(a.records) + (size_t)row * a.nblk + b);
-      m_b = r.x; s_b = r.y;
-    }
-    if (!(s_b > 0.f)) continue;                       // all -inf block
+  int best_i = -1;            // HIER / greedy: block number; FLAT: token id
+  auto merge = [&](int b, float m_b, float s_b, float flat_best, int flat_id) {
+    if (!(s_b > 0.f)) return;                         // all -inf block
     const float shift = (m_b - M) * a.inv_temp;
     const float rel = shift + logf(s_b);              // block log-sum-exp relative to M/T
     S += expf(rel);
@@ -294,19 +316,26 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
       const float sc = rel + gumbel_at(ds, 2u, (uint32_t)b);
       if (best_i < 0 || sc > best) { best = sc; best_i = b; }
     }
+  };
+  if (in_regs) {
+#pragma unroll
+    for (int i = 0; i < kRegRecords; ++i) {
+      const int b = lane + 32 * i;
+      if (b < a.nblk) {
+        if (SAMPLER == ESPO_SAMPLER_FLAT) merge(b, rm[i], rs[i], rf[i].z, __float_as_int(rf[i].w));
+        else merge(b, rm[i], rs[i], NINF, -1);
+      }
+    }
+  } else {
+    for (int b = lane; b < a.nblk; b += 32) {
+      float m_b, s_b, fb; int fi;
+      fetch(b, m_b, s_b, fb, fi);
+      merge(b, m_b, s_b, fb, fi);
+    }
   }
   S = warp_sum(S);
   warp_argmax(best, best_i);
-  if (best_i < 0) {   // no block offered a candidate: treat like an unusable row rather than index with -1
-    if (lane == 0) {
-      atomicOr(a.dev_status, ESPO_DEV_BAD_ROW);
-      a.status[slot] = ESPO_ROW_BAD;
-      a.tokens_out[row] = 0;
-      a.stop_out[row] = 0;
-      a.ticket[row] = 0;
-    }
-    return;
-  }
+  if (best_i < 0) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD); return; }   // nothing to pick from
 
   int token;
   float l_tok;
@@ -339,11 +368,7 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
 #pragma unroll
       for (int i = 0; i < kSubIds; ++i) x[i] = (i < n_here) ? load_logit<ES>(row_base, sub_lo + i) : NINF;
     }
-    float m_j = NINF;
-#pragma unroll
-    for (int i = 0; i < kSubIds; ++i) m_j = fmaxf(m_j, x[i]);
 
-    int sub_pick;
     if (a.greedy) {
       // first id equal to the maximum
       int first = -1;
@@ -351,10 +376,12 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
       for (int i = kSubIds - 1; i >= 0; --i) if (x[i] == M) first = sub_lo + i;
       float key = 0.f;
       warp_argmax(key, first);           // equal keys: lowest id wins
-      token = first;
+      token = max(first, blk_lo);
       l_tok = M;
-      sub_pick = -1;
     } else {
+      float m_j = NINF;
+#pragma unroll
+      for (int i = 0; i < kSubIds; ++i) m_j = fmaxf(m_j, x[i]);
       float sc = NINF;
       int j = -1;
       if (m_j > NINF) {
@@ -365,20 +392,23 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
         j = sub_lo >> 5;
       }
       warp_argmax(sc, j);
-      sub_pick = j;
-      // ---- ids of the chosen sub-block: lane e owns id 32*sub_pick + e ----
-      const int id = sub_pick * kSubIds + lane;
-      float sc0 = NINF, l = NINF;
-      int cand = -1;
-      if (id < a.V) {
-        l = load_logit<ES>(row_base, id);
-        if (l > NINF) { sc0 = (l - M) * a.inv_temp + gumbel_at(ds, 0u, (uint32_t)id); cand = id; }
+      const int sub_pick = max(j, blk_lo >> 5);        // j < 0 cannot happen: the block has a finite id
+      // ---- ids of the chosen sub-block: lane e takes id 32*sub_pick + e from the owning lane's registers ----
+      const int src = sub_pick & 31;
+      float mine = NINF;
+#pragma unroll
+      for (int i = 0; i < kSubIds; ++i) {
+        const float tv = __shfl_sync(kFullMask, x[i], src);
+        if (lane == i) mine = tv;
       }
+      const int id = sub_pick * kSubIds + lane;
+      float sc0 = NINF;
+      int cand = -1;
+      if (id < a.V && mine > NINF) { sc0 = (mine - M) * a.inv_temp + gumbel_at(ds, 0u, (uint32_t)id); cand = id; }
       warp_argmax(sc0, cand);
-      token = max(cand, sub_pick * kSubIds);   // cand < 0 cannot happen for a sub-block with a finite id
-      l_tok = __shfl_sync(kFullMask, l, token & 31);
+      token = max(cand, sub_pick * kSubIds);           // cand < 0 cannot happen for a sub-block with a finite id
+      l_tok = __shfl_sync(kFullMask, mine, token & 31);
     }
-    (void)sub_pick;
   } else {
     token = best_i;
     l_tok = load_logit<ES>(row_base, token);
@@ -390,10 +420,7 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
     const float logp = a.greedy ? 0.f : (-g - logf(S));
     float gt = (g - a.mu_g) * a.inv_sigma;
     gt = fminf(fmaxf(gt, -a.clip_c), a.clip_c);
-    const float z = fmaf(a.alpha_s, a.z[slot], a.one_minus_alpha * gt);
-    float v;
-    if (a.values_bf16) v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(a.values) + row) << 16);
-    else v = __ldg(reinterpret_cast<const float*>(a.values) + row);
+    const float z = fmaf(a.alpha_s, z_prev, a.one_minus_alpha * gt);
     const bool v_nan = (v != v);
     if (v_nan) atomicOr(a.dev_status, ESPO_DEV_NAN_VALUE);
     const float thr = a.beta * fmaxf(v, a.eps);
@@ -427,150 +454,194 @@ __device__ void finalize_row(const StepArgs& a, int row, int lane) {
 // The kernel.
 // -------------------------------------------------------------------------------------------
 
+// Where the CTA's range of the block sequence lies, in units local to the CTA: local block
+// index li = b0 + q for position q of the range; local row li / nblk; block li % nblk.
+struct CtaRange {
+  long long r_first;   // first row the range touches
+  int b0;              // block of that row at which the range starts
+  int n;               // blocks in the range
+  int off;             // walk order: position p of the walk is range position (p + off) mod n
+  int n_local;         // rows the range touches
+  int nblk;
+  __device__ __forceinline__ void locate(int p, int& lrow, int& blk) const {
+    int q = p + off;
+    if (q >= n) q -= n;
+    const int li = b0 + q;
+    lrow = li / nblk;
+    blk = li - lrow * nblk;
+  }
+  // blocks of local row k that belong to this CTA
+  __device__ __forceinline__ int share(int k) const { return min((k + 1) * nblk, b0 + n) - max(k * nblk, b0); }
+};
+
+// Take rows from the CTA's queue until none are left: add the CTA's share to the row's ticket
+// and finalize the row if that completed it.  Entry h is claimed before it is waited for, so
+// each entry is handled by exactly one warp.
+template <int ES, int SAMPLER>
+__device__ void drain_queue(const StepArgs& a, const CtaRange& cr, StepCtrl* ctrl, volatile int* queue,
+                            volatile int* cnt_unused, int lane) {
+  (void)cnt_unused;
+  volatile int* abort_flag = &ctrl->abort_flag;
+  for (;;) {
+    int h = 0;
+    if (lane == 0) h = atomicAdd(&ctrl->head, 1);
+    h = __shfl_sync(kFullMask, h, 0);
+    if (h >= cr.n_local) return;
+    int k = -1;
+    if (lane == 0) {
+      for (uint32_t it = 0; it < kPollSpinLimit; ++it) {
+        k = queue[h];
+        if (k >= 0 || *abort_flag) break;
+        __nanosleep(64);
+      }
+      if (k < 0 && !*abort_flag) { atomicOr(a.dev_status, ESPO_DEV_TIMEOUT); *abort_flag = 1; }
+    }
+    k = __shfl_sync(kFullMask, k, 0);
+    if (k < 0) return;
+    const int row = (int)(cr.r_first + k);
+    const unsigned share = (unsigned)cr.share(k);
+    unsigned old = 0;
+    if (lane == 0) {
+      __threadfence();                                   // the CTA's records before its ticket
+      old = atomicAdd(a.ticket + row, share);
+    }
+    old = __shfl_sync(kFullMask, old, 0);
+    if (old + share == (unsigned)a.nblk) {               // this CTA completed the row
+      __threadfence();
+      finalize_row<ES, SAMPLER>(a, row, lane);
+    }
+  }
+}
+
 template <int ES, int SAMPLER, bool BULK>
-__global__ void __launch_bounds__(kStepThreads) espo_step_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const StepArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
+  const int W = a.warps, S = a.stages;
   unsigned char* ring = smem;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)a.stages * a.tile_bytes);
-  uint64_t* empty_bar = full_bar + a.stages;
-  StepCtrl* ctrl = reinterpret_cast<StepCtrl*>(empty_bar + a.stages);
-  volatile int* queue = reinterpret_cast<volatile int*>(ctrl + 1);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)W * S * a.stage_bytes);
+  StepCtrl* ctrl = reinterpret_cast<StepCtrl*>(bars + W * S);
+  volatile int* cnt = reinterpret_cast<volatile int*>(ctrl + 1);
+  volatile int* queue = cnt + a.queue_cap;
   volatile int* abort_flag = &ctrl->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long t_begin = (long long)blockIdx.x * a.total_tiles / gridDim.x;
-  const long long t_end = (long long)(blockIdx.x + 1) * a.total_tiles / gridDim.x;
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < a.stages; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], kConsumerWarps);
-    }
-    ctrl->fin_tail = 0; ctrl->done_warps = 0; ctrl->abort_flag = 0; ctrl->pad = 0;
+  CtaRange cr;
+  {
+    const long long g0 = (long long)blockIdx.x * a.total_blocks / gridDim.x;
+    const long long g1 = (long long)(blockIdx.x + 1) * a.total_blocks / gridDim.x;
+    cr.nblk = a.nblk;
+    cr.r_first = g0 / a.nblk;
+    cr.b0 = (int)(g0 - cr.r_first * a.nblk);
+    cr.n = (int)(g1 - g0);
+    const long long r_last = (g1 - 1) / a.nblk;
+    cr.n_local = (int)(r_last - cr.r_first) + 1;
+    const long long last_start = r_last * a.nblk;       // the walk starts where the last row's part starts
+    cr.off = (last_start > g0) ? (int)(last_start - g0) : 0;
+  }
+
+  if (threadIdx.x == 0) { ctrl->head = 0; ctrl->posted = 0; ctrl->abort_flag = 0; ctrl->pad = 0; }
+  for (int i = threadIdx.x; i < a.queue_cap; i += blockDim.x) { cnt[i] = 0; queue[i] = -1; }
+  if (warp < W && lane == 0) {
+    for (int s = 0; s < S; ++s) mbar_init(&bars[warp * S + s], 1);
     mbar_init_fence();
   }
-  for (int i = threadIdx.x; i < a.queue_cap; i += blockDim.x) queue[i] = -1;
   __syncthreads();
 
-  if (warp < kConsumerWarps) {
-    // ------------------------------------------------------------------ consumers
-    int cur_row = -1;
-    unsigned cnt = 0;
+  if (warp < W) {
+    // ------------------------------------------------------------------ streaming warps
+    unsigned char* my_ring = ring + (size_t)warp * S * a.stage_bytes;
+    uint64_t* my_bar = bars + warp * S;
+    const int n_my = (cr.n > warp) ? (cr.n - warp + W - 1) / W : 0;
+
+    auto issue = [&](int i, int s) {   // lane 0: fetch the warp's i-th block into stage s
+      int lrow, blk;
+      cr.locate(warp + i * W, lrow, blk);
+      const uint32_t bytes = (uint32_t)min(kBlockIds, a.V - blk * kBlockIds) * ES;
+      const unsigned char* src = a.logits + (size_t)(cr.r_first + lrow) * a.row_stride_bytes + (size_t)blk * (kBlockIds * ES);
+      fence_proxy_async();             // the warp's reads of this stage come before the copy's writes
+      mbar_arrive_expect_tx(&my_bar[s], bytes);
+      bulk_copy_g2s(my_ring + (size_t)s * a.stage_bytes, src, bytes, &my_bar[s]);
+    };
+    if (BULK && lane == 0)
+      for (int i = 0; i < S && i < n_my; ++i) issue(i, i);
+
+    int cur_k = -1;
+    unsigned mine = 0;
     DrawStream ds{a.key0, a.key1, 0u, 0u, a.batch_bits};
     auto flush = [&]() {
-      if (lane == 0 && cnt > 0) {
-        __threadfence();                                      // records before the ticket
-        const unsigned old = atomicAdd(a.ticket + cur_row, cnt);
-        if (old + cnt == (unsigned)a.nblk) {                   // this warp completed the row
-          __threadfence();
-          const int qi = atomicAdd(&ctrl->fin_tail, 1);
-          if (qi < a.queue_cap) queue[qi] = cur_row;
-          else atomicOr(a.dev_status, ESPO_DEV_TIMEOUT);       // cannot happen: the host sizes the queue
+      if (lane == 0 && mine > 0) {
+        __threadfence_block();                                   // this warp's records before its count
+        const int old = atomicAdd(const_cast<int*>(cnt) + cur_k, (int)mine);
+        if (old + (int)mine == cr.share(cur_k)) {                // the CTA's share of the row is complete
+          __threadfence_block();
+          const int qi = atomicAdd(&ctrl->posted, 1);
+          if (qi < a.queue_cap) queue[qi] = cur_k;
+          else atomicOr(a.dev_status, ESPO_DEV_TIMEOUT);         // cannot happen: the host sizes the queue
         }
       }
-      cnt = 0;
+      mine = 0;
     };
+
     int s = 0;
     uint32_t parity = 0;
-    long long row = t_begin / a.tiles_per_row;
-    int tr = (int)(t_begin - row * a.tiles_per_row);
-    for (long long k = t_begin; k < t_end; ++k) {
-      if ((int)row != cur_row) {
+    int done = 0;
+    bool gave_up = false;
+    for (; done < n_my; ++done) {
+      int lrow, blk;
+      cr.locate(warp + done * W, lrow, blk);
+      if (lrow != cur_k) {
         flush();
-        cur_row = (int)row;
+        cur_k = lrow;
         if (SAMPLER == ESPO_SAMPLER_FLAT) {
           // the flat sampler perturbs every id, so the streaming warps need the row's draw stream
-          int slot = a.row_ids ? __ldg(a.row_ids + cur_row) : cur_row;
-          slot = min(max(slot, 0), a.capacity - 1);            // a bad slot is reported by the finalizer
+          const int row = (int)(cr.r_first + lrow);
+          int slot = a.row_ids ? __ldg(a.row_ids + row) : row;
+          slot = min(max(slot, 0), a.capacity - 1);              // a bad slot is reported by the finalizer
           ds.slot = (uint32_t)slot;
           ds.step = (uint32_t)a.t[slot];
         }
       }
-      if (!mbar_wait_bounded(&full_bar[s], parity, abort_flag)) {
-        if (lane == 0) { atomicOr(a.dev_status, ESPO_DEV_TIMEOUT); *abort_flag = 1; }
-        break;
-      }
-      const int block = tr * kConsumerWarps + warp;
-      if (block < a.nblk) {
-        const int nvalid = min(kBlockIds, a.V - block * kBlockIds);
-        reduce_block<ES, SAMPLER>(a, ring + (size_t)s * a.tile_bytes + (size_t)warp * (kBlockIds * ES), lane, nvalid,
-                                  cur_row, block, ds);
-        ++cnt;
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[s]);
-      if (++s == a.stages) { s = 0; parity ^= 1u; }
-      if (++tr == a.tiles_per_row) { tr = 0; ++row; }
-    }
-    flush();
-    if (lane == 0) { __threadfence_block(); atomicAdd(&ctrl->done_warps, 1); }
-  } else if (warp == kProducerWarp) {
-    // ------------------------------------------------------------------ producer
-    int s = 0;
-    uint32_t parity = 1;   // the first pass over the ring finds every stage free
-    bool first_round = true;
-    long long row = t_begin / a.tiles_per_row;
-    int tr = (int)(t_begin - row * a.tiles_per_row);
-    for (long long k = t_begin; k < t_end; ++k) {
-      if (!first_round) {
-        int ok = 1;
-        if (lane == 0) ok = mbar_wait_bounded(&empty_bar[s], parity, abort_flag) ? 1 : 0;
-        ok = __shfl_sync(kFullMask, ok, 0);
-        if (!ok) {
-          if (lane == 0) { atomicOr(a.dev_status, ESPO_DEV_TIMEOUT); *abort_flag = 1; }
-          break;
-        }
-      }
-      const int e0 = tr * kConsumerWarps * kBlockIds;
-      const int n = min(kConsumerWarps * kBlockIds, a.V - e0);
-      const unsigned char* src = a.logits + (size_t)row * a.row_stride_bytes + (size_t)e0 * ES;
-      unsigned char* dst = ring + (size_t)s * a.tile_bytes;
+      const int nvalid = min(kBlockIds, a.V - blk * kBlockIds);
+      const int row = (int)(cr.r_first + lrow);
+      unsigned char* stage = my_ring + (size_t)s * a.stage_bytes;
       if (BULK) {
-        if (lane == 0) {
-          mbar_arrive_expect_tx(&full_bar[s], (uint32_t)n * ES);
-          bulk_copy_g2s(dst, src, (uint32_t)n * ES, &full_bar[s]);
-        }
+        if (!mbar_wait_bounded(&my_bar[s], parity, abort_flag)) { gave_up = true; break; }
       } else {
+        // element-wise loader for rows that are not 16-byte aligned
+        const unsigned char* src = a.logits + (size_t)row * a.row_stride_bytes + (size_t)blk * (kBlockIds * ES);
         if (ES == 2) {
           const unsigned short* sp = reinterpret_cast<const unsigned short*>(src);
-          unsigned short* dp = reinterpret_cast<unsigned short*>(dst);
-          for (int i = lane; i < n; i += 32) dp[i] = __ldg(sp + i);
+          unsigned short* dp = reinterpret_cast<unsigned short*>(stage);
+          for (int i = lane; i < nvalid; i += 32) dp[i] = __ldg(sp + i);
         } else {
           const float* sp = reinterpret_cast<const float*>(src);
-          float* dp = reinterpret_cast<float*>(dst);
-          for (int i = lane; i < n; i += 32) dp[i] = __ldg(sp + i);
+          float* dp = reinterpret_cast<float*>(stage);
+          for (int i = lane; i < nvalid; i += 32) dp[i] = __ldg(sp + i);
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&full_bar[s]);
       }
-      if (++s == a.stages) { s = 0; first_round = false; parity ^= 1u; }
-      if (++tr == a.tiles_per_row) { tr = 0; ++row; }
+      reduce_block<ES, SAMPLER>(a, stage, lane, nvalid, row, blk, ds);
+      ++mine;
+      __syncwarp();
+      if (BULK) {
+        if (lane == 0 && done + S < n_my) issue(done + S, s);
+        if (++s == S) { s = 0; parity ^= 1u; }
+      }
     }
-    // The consumers wait for every copy issued above before they leave, and the CTA's
-    // shared memory outlives all of its warps, so nothing is in flight at exit.
-  } else {
-    // ------------------------------------------------------------------ finalizer
-    int head = 0;
-    for (;;) {
-      int row = -1;
-      bool finished = false, gave_up = true;
-      if (lane == 0) {
-        for (uint32_t it = 0; it < kPollSpinLimit; ++it) {
-          if (head < a.queue_cap && (row = queue[head]) >= 0) { gave_up = false; break; }
-          if (*(volatile int*)&ctrl->done_warps == kConsumerWarps && head >= *(volatile int*)&ctrl->fin_tail) { finished = true; gave_up = false; break; }
-          if (*abort_flag) { finished = true; gave_up = false; break; }
-          __nanosleep(100);
-        }
-        if (gave_up) { atomicOr(a.dev_status, ESPO_DEV_TIMEOUT); *abort_flag = 1; finished = true; }
+    if (gave_up) {
+      if (lane == 0) { atomicOr(a.dev_status, ESPO_DEV_TIMEOUT); *abort_flag = 1; }
+      // copies still in flight target this CTA's shared memory: give each one more bounded wait
+      for (int i = done; BULK && i < n_my && i < done + S; ++i) {
+        (void)mbar_wait_bounded(&my_bar[s], parity, nullptr);
+        if (++s == S) { s = 0; parity ^= 1u; }
       }
-      row = __shfl_sync(kFullMask, row, 0);
-      finished = __shfl_sync(kFullMask, finished, 0);
-      if (finished && row < 0) break;
-      __threadfence();
-      finalize_row<ES, SAMPLER>(a, row, lane);
-      ++head;
+    } else {
+      flush();
     }
   }
+  // The finalizer warp starts here at once; streaming warps join when they run out of blocks.
+  drain_queue<ES, SAMPLER>(a, cr, ctrl, queue, cnt, lane);
 }
 
 }  // namespace espo
@@ -582,7 +653,7 @@ __global__ void __launch_bounds__(kStepThreads) espo_step_kernel(const StepArgs 
 struct espo_state {
   int device, capacity, V, nblk, sm_count, max_smem;
   uint64_t seed, batch_id;
-  int cfg_stages, cfg_ctas_per_sm;   // 0 = library default
+  int cfg_warps, cfg_stages, cfg_ctas_per_sm;   // 0 = library default
   void* arena;
   size_t arena_bytes;
   float *z, *g, *g_tilde, *logp;
@@ -707,9 +778,12 @@ void espo_free_state(espo_state* st) {
   delete st;
 }
 
-int espo_set_launch_config(espo_state* st, int32_t stages, int32_t ctas_per_sm) {
+int espo_set_launch_config(espo_state* st, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm) {
   if (!st) return ESPO_ERR_NULL;
-  if (stages < 0 || stages > 64 || ctas_per_sm < 0 || ctas_per_sm > 8) return ESPO_ERR_BAD_PARAM;
+  if (consumer_warps < 0 || consumer_warps > espo::kMaxConsumerWarps || stages < 0 || stages > 64 || ctas_per_sm < 0 ||
+      ctas_per_sm > 8)
+    return ESPO_ERR_BAD_PARAM;
+  st->cfg_warps = consumer_warps;
   st->cfg_stages = stages;
   st->cfg_ctas_per_sm = ctas_per_sm;
   return ESPO_OK;
@@ -747,23 +821,30 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   a.row_ids = row_ids;
   a.n_rows = n_rows; a.V = st->V; a.capacity = st->capacity;
   a.nblk = st->nblk;
-  a.tiles_per_row = (st->nblk + kConsumerWarps - 1) / kConsumerWarps;
-  a.total_tiles = (long long)n_rows * a.tiles_per_row;
-  a.tile_bytes = kConsumerWarps * kBlockIds * es;
-  const int ctas_per_sm = st->cfg_ctas_per_sm ? st->cfg_ctas_per_sm : 2;
+  a.total_blocks = (long long)n_rows * st->nblk;
+  a.stage_bytes = kBlockIds * es;
+  // Launch shape: ctas_per_sm CTAs of `warps` streaming warps (+1 finalizer warp), `stages` blocks in flight per warp.
+  int ctas_per_sm = st->cfg_ctas_per_sm ? st->cfg_ctas_per_sm : (es == 2 ? 2 : 1);
+  int warps = st->cfg_warps ? st->cfg_warps : 15;
+  int stages = st->cfg_stages ? st->cfg_stages : 3;
+  if ((warps + 1) * 32 * ctas_per_sm > 2048) warps = 2048 / (32 * ctas_per_sm) - 1;
   long long grid = (long long)st->sm_count * ctas_per_sm;
-  if (grid > a.total_tiles) grid = a.total_tiles;
-  const long long tiles_per_cta = (a.total_tiles + grid - 1) / grid;
-  const long long qcap = tiles_per_cta / a.tiles_per_row + 2;
+  if (grid > a.total_blocks) grid = a.total_blocks;
+  const long long blocks_per_cta = (a.total_blocks + grid - 1) / grid;
+  if (blocks_per_cta < warps) warps = (int)blocks_per_cta;
+  const long long qcap = blocks_per_cta / a.nblk + 2;
   if (qcap > kMaxQueue) return ESPO_ERR_CAPACITY;
   a.queue_cap = (int)qcap;
-  const size_t fixed = sizeof(StepCtrl) + sizeof(int) * (size_t)a.queue_cap;
+  const size_t fixed = sizeof(StepCtrl) + 2 * sizeof(int) * (size_t)a.queue_cap;
   const size_t budget = (size_t)st->max_smem / ctas_per_sm - (ctas_per_sm > 1 ? 1024 : 0);
-  int stages = st->cfg_stages ? st->cfg_stages : (es == 2 ? 6 : 3);
-  while (stages > 1 && (size_t)stages * (a.tile_bytes + 16) + fixed > budget) --stages;
-  if (tiles_per_cta < stages) stages = (int)tiles_per_cta;
+  auto footprint = [&](int w, int sg) { return (size_t)w * sg * (a.stage_bytes + 8) + fixed; };
+  while (stages > 1 && footprint(warps, stages) > budget) --stages;
+  while (warps > 1 && footprint(warps, stages) > budget) --warps;
+  const long long per_warp = (blocks_per_cta + warps - 1) / warps;
+  if (per_warp < stages) stages = (int)per_warp;
+  a.warps = warps;
   a.stages = stages;
-  const size_t smem = (size_t)stages * (a.tile_bytes + 16) + fixed;
+  const size_t smem = footprint(warps, stages);
   if (smem > (size_t)st->max_smem) return ESPO_ERR_CAPACITY;
 
   a.z = st->z; a.g = st->g; a.g_tilde = st->g_tilde; a.logp = st->logp;
@@ -788,7 +869,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
 
   const bool bulk = ((uintptr_t)logits % 16 == 0) && (a.row_stride_bytes % 16 == 0) && (((size_t)st->V * es) % 16 == 0);
   StepKernel k = pick_kernel(es, p->sampler, bulk);
-  k<<<(unsigned)grid, kStepThreads, smem, (cudaStream_t)stream>>>(a);
+  k<<<(unsigned)grid, (unsigned)(warps + 1) * 32u, smem, (cudaStream_t)stream>>>(a);
   ESPO_CUDA_TRY(cudaGetLastError());
   return ESPO_OK;
 }

@@ -130,11 +130,11 @@ def test_results_do_not_depend_on_launch_shape_and_repeat_bit_exactly():
     x = synth.logits_batch(B, V, dtype=torch.bfloat16, seed=8)
     v = torch.rand(B, device="cuda")
     outs = []
-    for stages, ctas in [(0, 0), (0, 0), (2, 1), (4, 2), (3, 3), (12, 1)]:
+    for warps, stages, ctas in [(0, 0, 0), (0, 0, 0), (31, 2, 1), (8, 4, 2), (5, 3, 3), (1, 12, 1), (15, 1, 2)]:
         for sampler in SAMPLERS:
             p = espo.make_params(temperature=1.0, mu_g=1.0, sigma2_g=2.0, beta=2.0, sampler=sampler)
             st = espo.espo_init_state(B, V, seed=5)
-            espo.espo_set_launch_config(st, stages, ctas)
+            espo.espo_set_launch_config(st, warps, stages, ctas)
             tok = torch.empty(B, dtype=torch.int32, device="cuda")
             stop = torch.empty(B, dtype=torch.uint8, device="cuda")
             for _ in range(2):
