@@ -78,6 +78,29 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src_gm
       : "memory");
 }
 
+// ---------------------------------------------------------------- ordered global accesses
+
+// Adds to a counter in global memory; everything this thread wrote or observed before is
+// visible to whoever reads the new count with acquire semantics at device scope, and the
+// thread's later reads see what earlier adders published.
+__device__ __forceinline__ unsigned atom_add_acq_rel_gpu(unsigned* p, unsigned v) {
+  unsigned old;
+  asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+
+// Loads that are not served from the (incoherent) L1; the address may be shared or global.
+__device__ __forceinline__ float2 ld_volatile_f2(const void* p) {
+  float2 v;
+  asm volatile("ld.volatile.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ float4 ld_volatile_f4(const void* p) {
+  float4 v;
+  asm volatile("ld.volatile.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+  return v;
+}
+
 // ---------------------------------------------------------------- Philox4x32-10
 
 // Counter-based generator of Salmon et al. (SC'11): ten rounds, each two 32x32->64 multiplies
@@ -107,6 +130,12 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t word) {
   return -logf(-logf(u));
 }
 
+// The same uniform as a standard exponential draw E = -ln u > 0 (the Gumbel is -ln E).
+__device__ __forceinline__ float expo_from_word(uint32_t word) {
+  const float u = __uint2float_rn(2u * (word >> 9) + 1u) * 5.9604644775390625e-08f;
+  return -logf(u);
+}
+
 // Which Philox stream a draw belongs to: (step, slot, batch|level) are counter words 1..3.
 struct DrawStream {
   uint32_t k0, k1;     // seed halves
@@ -117,6 +146,11 @@ struct DrawStream {
 __device__ __forceinline__ float gumbel_at(const DrawStream& ds, uint32_t level, uint32_t index) {
   const uint4 w = philox4x32_10(index >> 2, ds.step, ds.slot, ds.batch_bits | level, ds.k0, ds.k1);
   return gumbel_from_word(pick_word(w, index & 3u));
+}
+
+__device__ __forceinline__ float expo_at(const DrawStream& ds, uint32_t level, uint32_t index) {
+  const uint4 w = philox4x32_10(index >> 2, ds.step, ds.slot, ds.batch_bits | level, ds.k0, ds.k1);
+  return expo_from_word(pick_word(w, index & 3u));
 }
 
 // ---------------------------------------------------------------- warp reductions

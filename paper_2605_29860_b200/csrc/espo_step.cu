@@ -42,7 +42,6 @@ namespace espo {
 constexpr int kMaxStepThreads = 1024;
 constexpr int kMaxConsumerWarps = kMaxStepThreads / 32 - 1;   // one more warp is the finalizer
 constexpr int kMaxQueue = 4096;
-constexpr int kRegRecords = 8;    // block records a finalizer lane keeps in registers (covers V <= 262144)
 
 struct StepArgs {
   // inputs
@@ -56,13 +55,15 @@ struct StepArgs {
   int nblk;                 // 1024-id blocks per row
   long long total_blocks;   // n_rows * nblk
   int warps, stages, stage_bytes, queue_cap;
+  int local_rows;           // rows whose block records fit in the CTA's shared-memory table (0: none)
+  int noise_rows;           // rows whose block-level noise fits in the CTA's shared-memory table
   // trajectory state (indexed by slot)
   float *z, *g, *g_tilde, *logp;
   int32_t *t, *t_stop;
   uint8_t* status;
   double *sum_g, *sum_g2;
   // scratch (indexed by row of this call)
-  float4* records;      // [capacity * nblk] block records (float2 view for the hierarchical sampler)
+  float4* records;      // [capacity * nblk] block records
   unsigned* ticket;     // [capacity] blocks of the row reduced so far
   unsigned* dev_status; // sticky ESPO_DEV_* bits
   // frozen parameters, pre-digested on the host
@@ -175,7 +176,7 @@ __device__ __forceinline__ int id_in_block(int j, int lane) {
 
 template <int ES, int SAMPLER>
 __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned char* blk, int lane, int nvalid,
-                                             int row, int block, const DrawStream& ds) {
+                                             void* rec_row, int block, const DrawStream& ds) {
   BlockVals<ES> bv;
   bv.load(blk, lane, nvalid);
   const float m_b = warp_max(bv.lane_max());
@@ -209,10 +210,9 @@ __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned c
       }
     }
     warp_argmax(best, best_id);
-    if (lane == 0)
-      a.records[(size_t)row * a.nblk + block] = make_float4(m_b, s_b, best, __int_as_float(best_id));
+    if (lane == 0) static_cast<float4*>(rec_row)[block] = make_float4(m_b, s_b, best, __int_as_float(best_id));
   } else {
-    if (lane == 0) reinterpret_cast<float2*>(a.records)[(size_t)row * a.nblk + block] = make_float2(m_b, s_b);
+    if (lane == 0) static_cast<float4*>(rec_row)[block] = make_float4(m_b, s_b, 0.f, 0.f);
   }
 }
 
@@ -227,7 +227,7 @@ __device__ __forceinline__ float load_logit(const unsigned char* row_base, int i
 }
 
 __device__ __forceinline__ void mark_row(const StepArgs& a, int row, int slot, int lane, int32_t token, unsigned dev_bit,
-                                         int new_status) {
+                                         int new_status, bool rec_local) {
   if (lane == 0) {
     if (dev_bit) atomicOr(a.dev_status, dev_bit);
     if (new_status >= 0) a.status[slot] = (uint8_t)new_status;
@@ -237,105 +237,101 @@ __device__ __forceinline__ void mark_row(const StepArgs& a, int row, int slot, i
   }
 }
 
+// What a finalizing warp reads about a row before it knows whether the row is complete: the
+// trajectory slot, its state, and the critic value.  Requested early so that the loads are in
+// flight while the row's ticket is being updated.
+struct __align__(16) RowPre {
+  int slot;         // -1: the row_ids entry was out of range
+  int status, t_now;
+  float z_prev, v;
+  double sum_g, sum_g2;
+};
+
+__device__ __forceinline__ RowPre prefetch_row(const StepArgs& a, int row) {
+  RowPre p;
+  p.slot = a.row_ids ? __ldg(a.row_ids + row) : row;
+  p.status = ESPO_ROW_ACTIVE; p.t_now = 0; p.z_prev = 0.f; p.sum_g = 0.0; p.sum_g2 = 0.0;
+  if (p.slot < 0 || p.slot >= a.capacity) {
+    p.slot = -1;
+  } else {
+    p.status = a.status[p.slot];
+    p.t_now = a.t[p.slot];
+    p.z_prev = a.z[p.slot];
+    p.sum_g = a.sum_g[p.slot];
+    p.sum_g2 = a.sum_g2[p.slot];
+  }
+  if (a.values_bf16) p.v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(a.values) + row) << 16);
+  else p.v = __ldg(reinterpret_cast<const float*>(a.values) + row);
+  return p;
+}
+
+// Sum over 32 values of 2^((x - m) * k2), two per packed multiply-add.
+__device__ __forceinline__ float sum_exp2_32(const float (&x)[kSubIds], float m, float k2) {
+  const float c0 = -m * k2;
+  const float2 k2v = make_float2(k2, k2), c0v = make_float2(c0, c0);
+  float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < kSubIds / 2; ++i) {
+    const float2 t = __ffma2_rn(make_float2(x[2 * i], x[2 * i + 1]), k2v, c0v);
+    const float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
+    if (i & 1) acc1 = __fadd2_rn(acc1, e); else acc0 = __fadd2_rn(acc0, e);
+  }
+  return (acc0.x + acc0.y) + (acc1.x + acc1.y);
+}
+
+// All perturbed scores below are "x/T + G" on the absolute scale of the logits, with the
+// Gumbel written through its exponential draw E = -ln u:  G = -ln E, and for a group with
+// log-sum-exp  m/T + ln s  the score is  m/T + ln(s / E).
 template <int ES, int SAMPLER>
-__device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane) {
+__device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, const RowPre pre, const void* rec_row,
+                                          bool rec_local, const float* noise) {
   const float NINF = __int_as_float(0xff800000);
-  const int slot = a.row_ids ? __ldg(a.row_ids + row) : row;
-  if (slot < 0 || slot >= a.capacity) { mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1); return; }
-  if (a.status[slot] != ESPO_ROW_ACTIVE) { mark_row(a, row, slot, lane, -1, 0u, -1); return; }   // finished: untouched
-
-  // per-trajectory state and the critic value: requested now, used at the very end
-  const int t_now = a.t[slot];
-  const float z_prev = a.z[slot];
-  float v;
-  if (a.values_bf16) v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(a.values) + row) << 16);
-  else v = __ldg(reinterpret_cast<const float*>(a.values) + row);
-
+  const int slot = pre.slot;
+  if (slot < 0) { mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, rec_local); return; }
+  if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, slot, lane, -1, 0u, -1, rec_local); return; }   // finished: untouched
+  const int t_now = pre.t_now;
   const unsigned char* row_base = a.logits + (size_t)row * a.row_stride_bytes;
   const DrawStream ds{a.key0, a.key1, (uint32_t)t_now, (uint32_t)slot, a.batch_bits};
 
-  // ---- the row's block records: lane l owns blocks l, l+32, ...; up to kRegRecords of them stay in registers ----
-  const bool in_regs = a.nblk <= 32 * kRegRecords;
-  float rm[kRegRecords], rs[kRegRecords];
-  float4 rf[SAMPLER == ESPO_SAMPLER_FLAT ? kRegRecords : 1];
-  auto fetch = [&](int b, float& m_b, float& s_b, float& fbest, int& fid) {
-    if (SAMPLER == ESPO_SAMPLER_FLAT) {
-      const float4 r = __ldcg(a.records + (size_t)row * a.nblk + b);
-      m_b = r.x; s_b = r.y; fbest = r.z; fid = __float_as_int(r.w);
-    } else {
-      const float2 r = __ldcg(reinterpret_cast<const float2*>(a.records) + (size_t)row * a.nblk + b);
-      m_b = r.x; s_b = r.y; fbest = NINF; fid = -1;
-    }
-  };
-  float M = NINF;
-  bool poisoned = false;
-  if (in_regs) {
-#pragma unroll
-    for (int i = 0; i < kRegRecords; ++i) {
-      const int b = lane + 32 * i;
-      rm[i] = NINF; rs[i] = 0.f;
-      if (SAMPLER == ESPO_SAMPLER_FLAT) rf[i] = make_float4(0.f, 0.f, NINF, __int_as_float(-1));
-      if (b < a.nblk) {
-        float fb; int fi;
-        fetch(b, rm[i], rs[i], fb, fi);
-        if (SAMPLER == ESPO_SAMPLER_FLAT) rf[i] = make_float4(0.f, 0.f, fb, __int_as_float(fi));
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < kRegRecords; ++i) {
-      M = fmaxf(M, rm[i]);
-      poisoned |= !(rs[i] >= 0.0f) || isinf(rs[i]);   // NaN or inf sum: the block held NaN or +inf
-    }
-  } else {
-    for (int b = lane; b < a.nblk; b += 32) {
-      float m_b, s_b, fb; int fi;
-      fetch(b, m_b, s_b, fb, fi);
-      M = fmaxf(M, m_b);
-      poisoned |= !(s_b >= 0.0f) || isinf(s_b);
-    }
-  }
-  M = warp_max(M);
-  poisoned = __any_sync(kFullMask, poisoned) || !(M > NINF) || isinf(M);
-  if (poisoned) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD); return; }
-
-  // ---- merge: S = sum_b s_b exp((m_b - M)/T); pick the block (HIER) or the id (FLAT) ----
-  float S = 0.f;              // lane-partial, summed below
-  float best = NINF;          // best perturbed score among this lane's blocks
+  // ---- one pass over the row's block records (m_b, s_b, third, fourth); lane l takes blocks l, l+32, ...
+  //      HIER: the block's perturbed score is m_b/T + ln s_b - ln E_b; `noise` (may be null) holds ln E_b
+  //      for every block of the row, prepared ahead of time by the CTA's finalizer warp;
+  //      FLAT: third = best perturbed score inside the block relative to m_b/T, fourth = its id.
+  //      Running (max, sum) per lane gives S = sum_b s_b exp((m_b - M)/T). ----
+  float run_m = NINF, run_s = 0.f;
+  float best = NINF;          // best perturbed score among this lane's blocks (greedy: largest block maximum)
   int best_i = -1;            // HIER / greedy: block number; FLAT: token id
-  auto merge = [&](int b, float m_b, float s_b, float flat_best, int flat_id) {
-    if (!(s_b > 0.f)) return;                         // all -inf block
-    const float shift = (m_b - M) * a.inv_temp;
-    const float rel = shift + logf(s_b);              // block log-sum-exp relative to M/T
-    S += expf(rel);
+  bool poisoned = false;
+  for (int b = lane; b < a.nblk; b += 32) {
+    const float4 r = ld_volatile_f4(static_cast<const float4*>(rec_row) + b);
+    const float m_b = r.x, s_b = r.y;
+    poisoned |= !(s_b >= 0.0f) || isinf(s_b);   // NaN or inf sum: the block held NaN or +inf
+    if (!(s_b > 0.f)) continue;                 // all -inf block
+    if (m_b > run_m) { run_s = fmaf(run_s, ex2_approx((run_m - m_b) * a.k2), s_b); run_m = m_b; }
+    else run_s = fmaf(s_b, ex2_approx((m_b - run_m) * a.k2), run_s);
     if (a.greedy) {
-      if (m_b == M && best_i < 0) { best = 0.f; best_i = b; }   // lowest block holding the maximum
+      if (m_b > best) { best = m_b; best_i = b; }                 // lowest block holding the maximum
     } else if (SAMPLER == ESPO_SAMPLER_FLAT) {
-      const float sc = flat_best + shift;
-      if (flat_id >= 0 && (best_i < 0 || sc > best)) { best = sc; best_i = flat_id; }
+      const float sc = fmaf(m_b, a.inv_temp, r.z);                // the block's best, moved to the absolute scale
+      const int id = __float_as_int(r.w);
+      if (id >= 0 && (best_i < 0 || sc > best)) { best = sc; best_i = id; }
     } else {
-      const float sc = rel + gumbel_at(ds, 2u, (uint32_t)b);
+      const float ln_e = noise ? noise[b] : logf(expo_at(ds, 2u, (uint32_t)b));
+      const float sc = fmaf(m_b, a.inv_temp, logf(s_b) - ln_e);
       if (best_i < 0 || sc > best) { best = sc; best_i = b; }
     }
-  };
-  if (in_regs) {
-#pragma unroll
-    for (int i = 0; i < kRegRecords; ++i) {
-      const int b = lane + 32 * i;
-      if (b < a.nblk) {
-        if (SAMPLER == ESPO_SAMPLER_FLAT) merge(b, rm[i], rs[i], rf[i].z, __float_as_int(rf[i].w));
-        else merge(b, rm[i], rs[i], NINF, -1);
-      }
-    }
-  } else {
-    for (int b = lane; b < a.nblk; b += 32) {
-      float m_b, s_b, fb; int fi;
-      fetch(b, m_b, s_b, fb, fi);
-      merge(b, m_b, s_b, fb, fi);
-    }
   }
-  S = warp_sum(S);
+  {
+    const float mm = warp_max(run_m);
+    if (run_m != mm) run_s *= ex2_approx((run_m - mm) * a.k2);   // run_m = -inf: run_s is 0 and stays 0
+    run_m = mm;
+    run_s = warp_sum(run_s);
+  }
+  const float M = run_m, S = run_s;
+  poisoned = __any_sync(kFullMask, poisoned) || !(M > NINF) || isinf(M);
+  if (poisoned) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, rec_local); return; }
   warp_argmax(best, best_i);
-  if (best_i < 0) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD); return; }   // nothing to pick from
+  if (best_i < 0) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, rec_local); return; }   // nothing to pick from
 
   int token;
   float l_tok;
@@ -385,11 +381,10 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane) 
       float sc = NINF;
       int j = -1;
       if (m_j > NINF) {
-        float s_j = 0.f;
-#pragma unroll
-        for (int i = 0; i < kSubIds; ++i) s_j += expf((x[i] - m_j) * a.inv_temp);
-        sc = (m_j - M) * a.inv_temp + logf(s_j) + gumbel_at(ds, 1u, (uint32_t)(sub_lo >> 5));
-        j = sub_lo >> 5;
+        const float s_j = sum_exp2_32(x, m_j, a.k2);
+        const uint32_t jg = (uint32_t)(sub_lo >> 5);   // global sub-block number
+        sc = fmaf(m_j, a.inv_temp, logf(s_j / expo_at(ds, 1u, jg)));
+        j = (int)jg;
       }
       warp_argmax(sc, j);
       const int sub_pick = max(j, blk_lo >> 5);        // j < 0 cannot happen: the block has a finite id
@@ -404,7 +399,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane) 
       const int id = sub_pick * kSubIds + lane;
       float sc0 = NINF;
       int cand = -1;
-      if (id < a.V && mine > NINF) { sc0 = (mine - M) * a.inv_temp + gumbel_at(ds, 0u, (uint32_t)id); cand = id; }
+      if (id < a.V && mine > NINF) { sc0 = fmaf(mine, a.inv_temp, -logf(expo_at(ds, 0u, (uint32_t)id))); cand = id; }
       warp_argmax(sc0, cand);
       token = max(cand, sub_pick * kSubIds);           // cand < 0 cannot happen for a sub-block with a finite id
       l_tok = __shfl_sync(kFullMask, mine, token & 31);
@@ -420,7 +415,8 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane) 
     const float logp = a.greedy ? 0.f : (-g - logf(S));
     float gt = (g - a.mu_g) * a.inv_sigma;
     gt = fminf(fmaxf(gt, -a.clip_c), a.clip_c);
-    const float z = fmaf(a.alpha_s, z_prev, a.one_minus_alpha * gt);
+    const float z = fmaf(a.alpha_s, pre.z_prev, a.one_minus_alpha * gt);
+    const float v = pre.v;
     const bool v_nan = (v != v);
     if (v_nan) atomicOr(a.dev_status, ESPO_DEV_NAN_VALUE);
     const float thr = a.beta * fmaxf(v, a.eps);
@@ -430,8 +426,8 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane) 
     a.g[slot] = g;
     a.g_tilde[slot] = gt;
     a.logp[slot] = logp;
-    a.sum_g[slot] += (double)g;
-    a.sum_g2[slot] += (double)g * (double)g;
+    a.sum_g[slot] = pre.sum_g + (double)g;
+    a.sum_g2[slot] = pre.sum_g2 + (double)g * (double)g;
     const int t_new = t_now + 1;
     a.t[slot] = t_new;
     uint8_t stop = 0;
@@ -446,7 +442,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane) 
     }
     a.tokens_out[row] = token;
     a.stop_out[row] = stop;
-    a.ticket[row] = 0;   // ready for the next launch
+    if (!rec_local) a.ticket[row] = 0;   // ready for the next launch
   }
 }
 
@@ -463,24 +459,34 @@ struct CtaRange {
   int off;             // walk order: position p of the walk is range position (p + off) mod n
   int n_local;         // rows the range touches
   int nblk;
-  __device__ __forceinline__ void locate(int p, int& lrow, int& blk) const {
-    int q = p + off;
-    if (q >= n) q -= n;
-    const int li = b0 + q;
-    lrow = li / nblk;
-    blk = li - lrow * nblk;
-  }
   // blocks of local row k that belong to this CTA
   __device__ __forceinline__ int share(int k) const { return min((k + 1) * nblk, b0 + n) - max(k * nblk, b0); }
+  // Rows that lie wholly inside the range need no other CTA: their records stay in shared memory.
+  // Such rows are consecutive, starting at local row (b0 == 0 ? 0 : 1); returns the table index or -1.
+  __device__ __forceinline__ int local_index(int k, int local_rows) const {
+    const int i = k - (b0 == 0 ? 0 : 1);
+    return (i >= 0 && i < local_rows && share(k) == nblk) ? i : -1;
+  }
+};
+
+// Take rows from the CTA's queue until none are left: add the CTA's share to the row's ticket
+// and finalize the row if that completed it.  Entry h is claimed before it is waited for, so
+// each entry is handled by exactly one warp.
+// Shared-memory tables a CTA keeps about the rows its range touches (indexed by local row).
+struct RowTables {
+  volatile int* queue;     // [queue_cap] local rows whose share of this CTA is complete, in completion order
+  volatile int* ready;     // [queue_cap] 1: pre[k] (and noise row k, if k < noise_rows) are filled in
+  RowPre* pre;             // [queue_cap]
+  float* noise;            // [noise_rows][nblk] ln E of the block-level draws (hierarchical sampler)
+  unsigned char* lrec;     // [local_rows][nblk] records of rows that lie wholly inside the range
 };
 
 // Take rows from the CTA's queue until none are left: add the CTA's share to the row's ticket
 // and finalize the row if that completed it.  Entry h is claimed before it is waited for, so
 // each entry is handled by exactly one warp.
 template <int ES, int SAMPLER>
-__device__ void drain_queue(const StepArgs& a, const CtaRange& cr, StepCtrl* ctrl, volatile int* queue,
-                            volatile int* cnt_unused, int lane) {
-  (void)cnt_unused;
+__device__ void drain_queue(const StepArgs& a, const CtaRange& cr, StepCtrl* ctrl, const RowTables& tb, int lane) {
+  constexpr int kRecBytes = 16;
   volatile int* abort_flag = &ctrl->abort_flag;
   for (;;) {
     int h = 0;
@@ -490,38 +496,92 @@ __device__ void drain_queue(const StepArgs& a, const CtaRange& cr, StepCtrl* ctr
     int k = -1;
     if (lane == 0) {
       for (uint32_t it = 0; it < kPollSpinLimit; ++it) {
-        k = queue[h];
+        k = tb.queue[h];
         if (k >= 0 || *abort_flag) break;
-        __nanosleep(64);
+        __nanosleep(32);
       }
       if (k < 0 && !*abort_flag) { atomicOr(a.dev_status, ESPO_DEV_TIMEOUT); *abort_flag = 1; }
+      __threadfence_block();                             // what the posting warp published before the entry
     }
     k = __shfl_sync(kFullMask, k, 0);
     if (k < 0) return;
     const int row = (int)(cr.r_first + k);
+    // the row's state and noise: from the tables if the finalizer warp got that far, else fetched here
+    const bool have = tb.ready[k] != 0;
+    __threadfence_block();
+    const RowPre pre = have ? tb.pre[k] : prefetch_row(a, row);
+    const float* noise = (have && SAMPLER == ESPO_SAMPLER_HIER && !a.greedy && k < a.noise_rows)
+                             ? tb.noise + (size_t)k * a.nblk : nullptr;
+    const int li = cr.local_index(k, a.local_rows);
+    if (li >= 0) {
+      // every record of the row was written by this CTA, into its shared-memory table
+      __syncwarp();
+      finalize_row<ES, SAMPLER>(a, row, lane, pre, tb.lrec + (size_t)li * a.nblk * kRecBytes, true, noise);
+      continue;
+    }
     const unsigned share = (unsigned)cr.share(k);
     unsigned old = 0;
-    if (lane == 0) {
-      __threadfence();                                   // the CTA's records before its ticket
-      old = atomicAdd(a.ticket + row, share);
-    }
+    if (lane == 0) old = atom_add_acq_rel_gpu(a.ticket + row, share);   // the CTA's records before its ticket
     old = __shfl_sync(kFullMask, old, 0);
-    if (old + share == (unsigned)a.nblk) {               // this CTA completed the row
-      __threadfence();
-      finalize_row<ES, SAMPLER>(a, row, lane);
+    __syncwarp();
+    if (old + share == (unsigned)a.nblk)                 // this CTA completed the row
+      finalize_row<ES, SAMPLER>(a, row, lane, pre,
+                                reinterpret_cast<const unsigned char*>(a.records) + (size_t)row * a.nblk * kRecBytes, false,
+                                noise);
+  }
+}
+
+// The finalizer warp's first job, while the streaming warps fetch their first blocks: read the
+// state of every row the range touches and draw the block-level noise of those rows.
+template <int SAMPLER>
+__device__ void prepare_rows(const StepArgs& a, const CtaRange& cr, const RowTables& tb, int lane) {
+  for (int k = 0; k < cr.n_local; ++k) {
+    const int row = (int)(cr.r_first + k);
+    const RowPre pre = prefetch_row(a, row);
+    if (lane == 0) tb.pre[k] = pre;
+    if (SAMPLER == ESPO_SAMPLER_HIER && !a.greedy && k < a.noise_rows && pre.slot >= 0 && pre.status == ESPO_ROW_ACTIVE) {
+      const DrawStream ds{a.key0, a.key1, (uint32_t)pre.t_now, (uint32_t)pre.slot, a.batch_bits};
+      // lane l draws for blocks 4l..4l+3 of every group of 128: one Philox call serves four blocks
+      for (int c0 = 0; c0 < a.nblk; c0 += 128) {
+        const int b0 = c0 + 4 * lane;
+        if (b0 >= a.nblk) continue;
+        const uint4 rnd = philox4x32_10((uint32_t)b0 >> 2, ds.step, ds.slot, ds.batch_bits | 2u, ds.k0, ds.k1);
+        const uint32_t wd[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (b0 + i < a.nblk) tb.noise[(size_t)k * a.nblk + b0 + i] = logf(expo_from_word(wd[i]));
+      }
     }
+    __syncwarp();
+    if (lane == 0) { __threadfence_block(); tb.ready[k] = 1; }
   }
 }
 
 template <int ES, int SAMPLER, bool BULK>
-__global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __grid_constant__ StepArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int W = a.warps, S = a.stages;
   unsigned char* ring = smem;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)W * S * a.stage_bytes);
-  StepCtrl* ctrl = reinterpret_cast<StepCtrl*>(bars + W * S);
+  int2* metas = reinterpret_cast<int2*>(bars + W * S);
+  StepCtrl* ctrl = reinterpret_cast<StepCtrl*>(metas + W * S);
   volatile int* cnt = reinterpret_cast<volatile int*>(ctrl + 1);
-  volatile int* queue = cnt + a.queue_cap;
+  RowTables tb;
+  tb.queue = cnt + a.queue_cap;
+  tb.ready = tb.queue + a.queue_cap;
+  {
+    // 16-byte aligned tables after the int arrays
+    size_t off = (size_t)W * S * (a.stage_bytes + 16) + sizeof(StepCtrl) + 3 * sizeof(int) * (size_t)a.queue_cap;
+    off = (off + 15) & ~(size_t)15;
+    tb.pre = reinterpret_cast<RowPre*>(smem + off);
+    off += sizeof(RowPre) * (size_t)a.queue_cap;
+    tb.noise = reinterpret_cast<float*>(smem + off);
+    off += ((sizeof(float) * (size_t)a.noise_rows * a.nblk) + 15) & ~(size_t)15;
+    tb.lrec = smem + off;
+  }
+  volatile int* queue = tb.queue;
+  unsigned char* lrec = tb.lrec;
+  constexpr int kRecBytes = 16;
   volatile int* abort_flag = &ctrl->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -541,7 +601,7 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const Ste
   }
 
   if (threadIdx.x == 0) { ctrl->head = 0; ctrl->posted = 0; ctrl->abort_flag = 0; ctrl->pad = 0; }
-  for (int i = threadIdx.x; i < a.queue_cap; i += blockDim.x) { cnt[i] = 0; queue[i] = -1; }
+  for (int i = threadIdx.x; i < a.queue_cap; i += blockDim.x) { cnt[i] = 0; tb.queue[i] = -1; tb.ready[i] = 0; }
   if (warp < W && lane == 0) {
     for (int s = 0; s < S; ++s) mbar_init(&bars[warp * S + s], 1);
     mbar_init_fence();
@@ -552,22 +612,55 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const Ste
     // ------------------------------------------------------------------ streaming warps
     unsigned char* my_ring = ring + (size_t)warp * S * a.stage_bytes;
     uint64_t* my_bar = bars + warp * S;
+    int2* my_meta = metas + warp * S;            // (local row, block) of the block each stage holds
     const int n_my = (cr.n > warp) ? (cr.n - warp + W - 1) / W : 0;
+    constexpr int kBlockBytes = kBlockIds * ES;
 
-    auto issue = [&](int i, int s) {   // lane 0: fetch the warp's i-th block into stage s
-      int lrow, blk;
-      cr.locate(warp + i * W, lrow, blk);
-      const uint32_t bytes = (uint32_t)min(kBlockIds, a.V - blk * kBlockIds) * ES;
-      const unsigned char* src = a.logits + (size_t)(cr.r_first + lrow) * a.row_stride_bytes + (size_t)blk * (kBlockIds * ES);
+    // Where the warp's next block to fetch lies.  The warp takes every W-th position of the CTA's walk, so the
+    // cursor moves by W blocks at a time and only divides when the walk wraps around the end of the range.
+    int fq, f_lrow, f_blk;
+    const unsigned char* f_ptr;
+    auto seek = [&](int q) {
+      fq = q;
+      const int li = cr.b0 + q;
+      f_lrow = li / cr.nblk;
+      f_blk = li - f_lrow * cr.nblk;
+      f_ptr = a.logits + (size_t)(cr.r_first + f_lrow) * a.row_stride_bytes + (size_t)f_blk * kBlockBytes;
+    };
+    auto advance = [&]() {
+      fq += W;
+      if (fq >= cr.n) { seek(fq - cr.n); return; }
+      f_blk += W;
+      f_ptr += (size_t)W * kBlockBytes;
+      while (f_blk >= cr.nblk) {
+        f_blk -= cr.nblk;
+        ++f_lrow;
+        f_ptr += a.row_stride_bytes - (int64_t)cr.nblk * kBlockBytes;
+      }
+    };
+    {
+      int q = warp + cr.off;
+      if (q >= cr.n) q -= cr.n;
+      seek(n_my > 0 ? q : 0);
+    }
+    auto issue = [&](int s) {   // lane 0: fetch the block under the cursor into stage s
+      const uint32_t bytes = (uint32_t)min(kBlockIds, a.V - f_blk * kBlockIds) * ES;
+      my_meta[s] = make_int2(f_lrow, f_blk);
       fence_proxy_async();             // the warp's reads of this stage come before the copy's writes
       mbar_arrive_expect_tx(&my_bar[s], bytes);
-      bulk_copy_g2s(my_ring + (size_t)s * a.stage_bytes, src, bytes, &my_bar[s]);
+      bulk_copy_g2s(my_ring + (size_t)s * a.stage_bytes, f_ptr, bytes, &my_bar[s]);
     };
-    if (BULK && lane == 0)
-      for (int i = 0; i < S && i < n_my; ++i) issue(i, i);
+    int fetched = 0;
+    if (BULK) {
+      for (; fetched < S && fetched < n_my; ++fetched) {
+        if (lane == 0) issue(fetched);
+        advance();
+      }
+    }
 
     int cur_k = -1;
     unsigned mine = 0;
+    void* rec_row = nullptr;
     DrawStream ds{a.key0, a.key1, 0u, 0u, a.batch_bits};
     auto flush = [&]() {
       if (lane == 0 && mine > 0) {
@@ -588,11 +681,37 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const Ste
     int done = 0;
     bool gave_up = false;
     for (; done < n_my; ++done) {
+      unsigned char* stage = my_ring + (size_t)s * a.stage_bytes;
       int lrow, blk;
-      cr.locate(warp + done * W, lrow, blk);
+      if (BULK) {
+        if (!mbar_wait_bounded(&my_bar[s], parity, abort_flag)) { gave_up = true; break; }
+        const int2 mt = my_meta[s];
+        lrow = mt.x; blk = mt.y;
+      } else {
+        lrow = f_lrow; blk = f_blk;
+      }
+      const int nvalid = min(kBlockIds, a.V - blk * kBlockIds);
+      if (!BULK) {
+        // element-wise loader for rows that are not 16-byte aligned
+        if (ES == 2) {
+          const unsigned short* sp = reinterpret_cast<const unsigned short*>(f_ptr);
+          unsigned short* dp = reinterpret_cast<unsigned short*>(stage);
+          for (int i = lane; i < nvalid; i += 32) dp[i] = __ldg(sp + i);
+        } else {
+          const float* sp = reinterpret_cast<const float*>(f_ptr);
+          float* dp = reinterpret_cast<float*>(stage);
+          for (int i = lane; i < nvalid; i += 32) dp[i] = __ldg(sp + i);
+        }
+        advance();
+        __syncwarp();
+      }
       if (lrow != cur_k) {
         flush();
         cur_k = lrow;
+        const int li = cr.local_index(lrow, a.local_rows);
+        rec_row = (li >= 0) ? static_cast<void*>(lrec + (size_t)li * a.nblk * kRecBytes)
+                            : static_cast<void*>(reinterpret_cast<unsigned char*>(a.records) +
+                                                 (size_t)(cr.r_first + lrow) * a.nblk * kRecBytes);
         if (SAMPLER == ESPO_SAMPLER_FLAT) {
           // the flat sampler perturbs every id, so the streaming warps need the row's draw stream
           const int row = (int)(cr.r_first + lrow);
@@ -602,37 +721,22 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const Ste
           ds.step = (uint32_t)a.t[slot];
         }
       }
-      const int nvalid = min(kBlockIds, a.V - blk * kBlockIds);
-      const int row = (int)(cr.r_first + lrow);
-      unsigned char* stage = my_ring + (size_t)s * a.stage_bytes;
-      if (BULK) {
-        if (!mbar_wait_bounded(&my_bar[s], parity, abort_flag)) { gave_up = true; break; }
-      } else {
-        // element-wise loader for rows that are not 16-byte aligned
-        const unsigned char* src = a.logits + (size_t)row * a.row_stride_bytes + (size_t)blk * (kBlockIds * ES);
-        if (ES == 2) {
-          const unsigned short* sp = reinterpret_cast<const unsigned short*>(src);
-          unsigned short* dp = reinterpret_cast<unsigned short*>(stage);
-          for (int i = lane; i < nvalid; i += 32) dp[i] = __ldg(sp + i);
-        } else {
-          const float* sp = reinterpret_cast<const float*>(src);
-          float* dp = reinterpret_cast<float*>(stage);
-          for (int i = lane; i < nvalid; i += 32) dp[i] = __ldg(sp + i);
-        }
-        __syncwarp();
-      }
-      reduce_block<ES, SAMPLER>(a, stage, lane, nvalid, row, blk, ds);
+      reduce_block<ES, SAMPLER>(a, stage, lane, nvalid, rec_row, blk, ds);
       ++mine;
       __syncwarp();
       if (BULK) {
-        if (lane == 0 && done + S < n_my) issue(done + S, s);
+        if (fetched < n_my) {
+          if (lane == 0) issue(s);
+          advance();
+          ++fetched;
+        }
         if (++s == S) { s = 0; parity ^= 1u; }
       }
     }
     if (gave_up) {
       if (lane == 0) { atomicOr(a.dev_status, ESPO_DEV_TIMEOUT); *abort_flag = 1; }
       // copies still in flight target this CTA's shared memory: give each one more bounded wait
-      for (int i = done; BULK && i < n_my && i < done + S; ++i) {
+      for (int i = done; BULK && i < fetched; ++i) {
         (void)mbar_wait_bounded(&my_bar[s], parity, nullptr);
         if (++s == S) { s = 0; parity ^= 1u; }
       }
@@ -640,8 +744,9 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const Ste
       flush();
     }
   }
-  // The finalizer warp starts here at once; streaming warps join when they run out of blocks.
-  drain_queue<ES, SAMPLER>(a, cr, ctrl, queue, cnt, lane);
+  // The finalizer warp comes here at once; streaming warps join when they run out of blocks.
+  if (warp == W) prepare_rows<SAMPLER>(a, cr, tb, lane);
+  drain_queue<ES, SAMPLER>(a, cr, ctrl, tb, lane);
 }
 
 }  // namespace espo
@@ -824,9 +929,9 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   a.total_blocks = (long long)n_rows * st->nblk;
   a.stage_bytes = kBlockIds * es;
   // Launch shape: ctas_per_sm CTAs of `warps` streaming warps (+1 finalizer warp), `stages` blocks in flight per warp.
-  int ctas_per_sm = st->cfg_ctas_per_sm ? st->cfg_ctas_per_sm : (es == 2 ? 2 : 1);
-  int warps = st->cfg_warps ? st->cfg_warps : 15;
-  int stages = st->cfg_stages ? st->cfg_stages : 3;
+  int ctas_per_sm = st->cfg_ctas_per_sm ? st->cfg_ctas_per_sm : 1;
+  int warps = st->cfg_warps ? st->cfg_warps : (es == 2 ? 31 : 15);
+  int stages = st->cfg_stages ? st->cfg_stages : 2;
   if ((warps + 1) * 32 * ctas_per_sm > 2048) warps = 2048 / (32 * ctas_per_sm) - 1;
   long long grid = (long long)st->sm_count * ctas_per_sm;
   if (grid > a.total_blocks) grid = a.total_blocks;
@@ -835,9 +940,19 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   const long long qcap = blocks_per_cta / a.nblk + 2;
   if (qcap > kMaxQueue) return ESPO_ERR_CAPACITY;
   a.queue_cap = (int)qcap;
-  const size_t fixed = sizeof(StepCtrl) + 2 * sizeof(int) * (size_t)a.queue_cap;
+  // shared-memory table for the records of rows that one CTA reduces alone (at most 16 KB of it)
+  const size_t rec_bytes = (size_t)a.nblk * 16;
+  long long local_rows = blocks_per_cta / a.nblk + 1;
+  if ((size_t)local_rows * rec_bytes > 16384) local_rows = (long long)(16384 / rec_bytes);
+  a.local_rows = (int)local_rows;
+  // ... and one for the block-level noise of the rows the range touches (at most 16 KB)
+  long long noise_rows = a.queue_cap;
+  if ((size_t)noise_rows * a.nblk * 4 > 16384) noise_rows = (long long)(16384 / ((size_t)a.nblk * 4));
+  a.noise_rows = (int)noise_rows;
+  const size_t fixed = sizeof(StepCtrl) + 3 * sizeof(int) * (size_t)a.queue_cap + 16 + sizeof(RowPre) * (size_t)a.queue_cap +
+                       (((size_t)a.noise_rows * a.nblk * 4 + 15) & ~(size_t)15) + (size_t)a.local_rows * rec_bytes;
   const size_t budget = (size_t)st->max_smem / ctas_per_sm - (ctas_per_sm > 1 ? 1024 : 0);
-  auto footprint = [&](int w, int sg) { return (size_t)w * sg * (a.stage_bytes + 8) + fixed; };
+  auto footprint = [&](int w, int sg) { return (size_t)w * sg * (a.stage_bytes + 16) + fixed; };
   while (stages > 1 && footprint(warps, stages) > budget) --stages;
   while (warps > 1 && footprint(warps, stages) > budget) --warps;
   const long long per_warp = (blocks_per_cta + warps - 1) / warps;
