@@ -78,6 +78,13 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src_gm
       : "memory");
 }
 
+// Barrier 1 of the CTA, for `threads` threads (a multiple of 32): warps running different code
+// (streaming warps, the finalizer warp) meet here once; unlike __syncthreads() it may be reached
+// from different places in the program.
+__device__ __forceinline__ void cta_rendezvous(unsigned threads) {
+  asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory");
+}
+
 // ---------------------------------------------------------------- ordered global accesses
 
 // Adds to a counter in global memory; everything this thread wrote or observed before is

@@ -298,17 +298,17 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
   //      for every block of the row, prepared ahead of time by the CTA's finalizer warp;
   //      FLAT: third = best perturbed score inside the block relative to m_b/T, fourth = its id.
   //      Running (max, sum) per lane gives S = sum_b s_b exp((m_b - M)/T). ----
-  float run_m = NINF, run_s = 0.f;
   float best = NINF;          // best perturbed score among this lane's blocks (greedy: largest block maximum)
   int best_i = -1;            // HIER / greedy: block number; FLAT: token id
   bool poisoned = false;
-  for (int b = lane; b < a.nblk; b += 32) {
-    const float4 r = ld_volatile_f4(static_cast<const float4*>(rec_row) + b);
+  float run_m = NINF, run_s = 0.f;
+  auto load_rec = [&](int b) -> float4 {
+    const float4* rp = static_cast<const float4*>(rec_row) + b;
+    return rec_local ? *rp : __ldcg(rp);       // shared-memory table, or global records written by other CTAs
+  };
+  auto score = [&](int b, const float4& r) {
     const float m_b = r.x, s_b = r.y;
-    poisoned |= !(s_b >= 0.0f) || isinf(s_b);   // NaN or inf sum: the block held NaN or +inf
-    if (!(s_b > 0.f)) continue;                 // all -inf block
-    if (m_b > run_m) { run_s = fmaf(run_s, ex2_approx((run_m - m_b) * a.k2), s_b); run_m = m_b; }
-    else run_s = fmaf(s_b, ex2_approx((m_b - run_m) * a.k2), run_s);
+    if (!(s_b > 0.f)) return;                   // all -inf block
     if (a.greedy) {
       if (m_b > best) { best = m_b; best_i = b; }                 // lowest block holding the maximum
     } else if (SAMPLER == ESPO_SAMPLER_FLAT) {
@@ -320,6 +320,29 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       const float sc = fmaf(m_b, a.inv_temp, logf(s_b) - ln_e);
       if (best_i < 0 || sc > best) { best = sc; best_i = b; }
     }
+  };
+  constexpr int kPerLane = 5;                   // records a lane holds at once (covers V <= 163840 in one go)
+  for (int base = 0; base < a.nblk; base += 32 * kPerLane) {
+    float4 r[kPerLane];
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+      const int b = base + 32 * i + lane;
+      r[i] = (b < a.nblk) ? load_rec(b) : make_float4(NINF, 0.f, NINF, __int_as_float(-1));
+    }
+    float lm = run_m;
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+      poisoned |= !(r[i].y >= 0.0f) || isinf(r[i].y);   // NaN or inf sum: the block held NaN or +inf
+      if (r[i].y > 0.f) lm = fmaxf(lm, r[i].x);
+    }
+    // sum of s_b 2^((m_b - lm) k2), independent terms; the carried sum is rescaled once
+    float acc = (run_m == lm) ? run_s : run_s * ex2_approx((run_m - lm) * a.k2);
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i)
+      if (r[i].y > 0.f) acc = fmaf(r[i].y, ex2_approx((r[i].x - lm) * a.k2), acc);
+    run_m = lm; run_s = acc;
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) score(base + 32 * i + lane, r[i]);
   }
   {
     const float mm = warp_max(run_m);
@@ -328,6 +351,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
     run_s = warp_sum(run_s);
   }
   const float M = run_m, S = run_s;
+  const float log_S = logf(S);   // needed at the very end; started before the loads below
   poisoned = __any_sync(kFullMask, poisoned) || !(M > NINF) || isinf(M);
   if (poisoned) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, rec_local); return; }
   warp_argmax(best, best_i);
@@ -412,7 +436,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
   if (lane == 0) {
     // Eq. 5: the normaliser cancels; Eq. 8; Eq. 9; Eq. 10.
     const float g = a.greedy ? 0.f : (M - l_tok) * a.inv_temp;
-    const float logp = a.greedy ? 0.f : (-g - logf(S));
+    const float logp = a.greedy ? 0.f : (-g - log_S);
     float gt = (g - a.mu_g) * a.inv_sigma;
     gt = fminf(fmaxf(gt, -a.clip_c), a.clip_c);
     const float z = fmaf(a.alpha_s, pre.z_prev, a.one_minus_alpha * gt);
@@ -606,7 +630,9 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
     for (int s = 0; s < S; ++s) mbar_init(&bars[warp * S + s], 1);
     mbar_init_fence();
   }
-  __syncthreads();
+  __syncwarp();
+  // A streaming warp needs only its own barriers to start fetching; the CTA-wide tables set up above are first
+  // touched after the rendezvous (A) that follows the first fetches.
 
   if (warp < W) {
     // ------------------------------------------------------------------ streaming warps
@@ -657,6 +683,7 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
         advance();
       }
     }
+    cta_rendezvous(blockDim.x);   // (A) the queue, counters and tables are initialised
 
     int cur_k = -1;
     unsigned mine = 0;
@@ -745,7 +772,10 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
     }
   }
   // The finalizer warp comes here at once; streaming warps join when they run out of blocks.
-  if (warp == W) prepare_rows<SAMPLER>(a, cr, tb, lane);
+  if (warp == W) {
+    cta_rendezvous(blockDim.x);   // (A)
+    prepare_rows<SAMPLER>(a, cr, tb, lane);
+  }
   drain_queue<ES, SAMPLER>(a, cr, ctrl, tb, lane);
 }
 
