@@ -10,7 +10,8 @@ K*B tokens that rollout generated -- the whole path, at the cadence the method r
 The advantage kernel is additionally timed on its own workload (1024 ragged trajectories of
 256..16384 tokens) and reported under "advantage_pass".
 
-Prints one JSON line (see the design doc for the field-by-field definition).
+Prints one JSON line: the metric, the roofline of the step kernel, the advantage pass, an end-to-end figure with
+host buffers, sampled clocks and the CPU oracle timed on the same box.
 """
 from __future__ import annotations
 
@@ -178,6 +179,7 @@ def main():
     ap.add_argument("--rows", type=int, default=B_ROWS, help="rollout batch size B (default: the headline 512)")
     ap.add_argument("--sampler", default="hier", choices=["hier", "flat"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the single-step timings at other shapes")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = args.steps or 4
@@ -314,6 +316,37 @@ def main():
                          "traffic": None, "bytes_per_token": 12},
         }
         del r, v, L, s, a_out
+
+        # ---- single-step bandwidth at other shapes (the large-batch sweep; rotating buffers larger than 2x L2) ----
+        if not args.no_sweep:
+            sweep = []
+            for (sB, sV, sdt) in ((256, VOCAB, torch.bfloat16), (1024, VOCAB, torch.bfloat16), (2048, VOCAB, torch.bfloat16),
+                                  (512, VOCAB, torch.float32), (512, 128256, torch.bfloat16), (2048, 32000, torch.bfloat16)):
+                es = 2 if sdt == torch.bfloat16 else 4
+                per = sB * sV * es
+                nb = max(2, int(280e6 // per) + 1)
+                sbufs = [synth.logits_batch(sB, sV, dtype=sdt, sd=3.0, seed=500 + i, device=dev) for i in range(nb)]
+                sst = espo.espo_init_state(sB, sV, seed=99)
+                sval = torch.full((sB,), 0.5, dtype=torch.bfloat16, device=dev)
+                stok = torch.empty(sB, dtype=torch.int32, device=dev)
+                sstop = torch.empty(sB, dtype=torch.uint8, device=dev)
+                for i in range(20):
+                    espo.espo_step(sbufs[i % nb], sval, sst, params, stok, sstop)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                reps = 200
+                e0.record()
+                for i in range(reps):
+                    espo.espo_step(sbufs[i % nb], sval, sst, params, stok, sstop)
+                e1.record()
+                torch.cuda.synchronize()
+                us = e0.elapsed_time(e1) * 1e3 / reps
+                gbs = per / us / 1e3
+                sweep.append({"B": sB, "V": sV, "logits": "bf16" if es == 2 else "f32", "us": us, "GB/s": gbs,
+                              "frac_of_measured_peak": gbs / peak, "rows/s": sB / (us * 1e-6)})
+                espo.espo_free_state(sst)
+                del sbufs
+            out["bandwidth_sweep"] = sweep
 
         # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region ----
         host_logits = [torch.empty(B, V, dtype=torch.bfloat16).pin_memory() for _ in range(2)]

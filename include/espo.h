@@ -8,10 +8,10 @@
  *
  *   espo_step        one pass of the rollout loop body (Algorithm 1) over a batch of
  *                    logit rows: log-softmax statistics, Philox Gumbel-max sampling,
- *                    surrogate regret (Eq. 5), normalisation (Eq. 8), smoothing (Eq. 9),
- *                    value-gated stop test (Eq. 10), per-trajectory bookkeeping;
- *   espo_advantages  TD errors and GAE (Eq. 3-4) over ragged truncated trajectories with
- *                    the failure transition of Eq. 12.
+ *                    surrogate regret (Eq. 6), normalisation (Eq. 9), smoothing (Eq. 10),
+ *                    value-gated stop test (Eq. 11), per-trajectory bookkeeping;
+ *   espo_advantages  TD errors and GAE (Eq. 4-5) over ragged truncated trajectories with
+ *                    the failure transition of Eq. 13.
  *
  * Conventions for every entry point
  *   - "device" pointers are CUDA device memory owned by the caller, on the device that
@@ -60,7 +60,7 @@ extern "C" {
 
 /* ---- per-trajectory status (espo_state_view: status[]) ------------------------------ */
 #define ESPO_ROW_ACTIVE   0
-#define ESPO_ROW_STOPPED  1   /* ESPO's rule fired (Eq. 10): failure transition            */
+#define ESPO_ROW_STOPPED  1   /* ESPO's rule fired (Eq. 11): failure transition            */
 #define ESPO_ROW_EOS      2   /* sampled the end-of-sequence token                          */
 #define ESPO_ROW_TMAX     3   /* reached the horizon t_max                                  */
 #define ESPO_ROW_BAD      4   /* the logit row held NaN / +inf, or no finite entry          */
@@ -76,13 +76,13 @@ extern "C" {
  * only updated at batch boundaries).  Plain data, passed by host pointer, copied at call. */
 typedef struct espo_params {
   float   temperature;      /* > 0 samples from softmax(logits/temperature); 0 = greedy    */
-  float   mu_g;             /* running mean of the regret, Eq. 6                            */
-  float   sigma2_g;         /* running variance of the regret, Eq. 7 (>= 0)                 */
-  float   delta;            /* stabiliser under the square root in Eq. 8 (sigma2_g+delta>0) */
-  float   clip_c;           /* clipping bound c of Eq. 8 (> 0)                              */
-  float   alpha_s;          /* smoothing factor of Eq. 9, in [0, 1)                         */
-  float   beta;             /* threshold multiplier of Eq. 10                               */
-  float   eps;              /* value floor epsilon of Eq. 10                                */
+  float   mu_g;             /* running mean of the regret, Eq. 7                            */
+  float   sigma2_g;         /* running variance of the regret, Eq. 8 (>= 0)                 */
+  float   delta;            /* stabiliser under the square root in Eq. 9 (sigma2_g+delta>0) */
+  float   clip_c;           /* clipping bound c of Eq. 9 (> 0)                              */
+  float   alpha_s;          /* smoothing factor of Eq. 10, in [0, 1)                         */
+  float   beta;             /* threshold multiplier of Eq. 11                               */
+  float   eps;              /* value floor epsilon of Eq. 11                                */
   int32_t warmup_complete;  /* 0: the stop test is disabled (critic warm-up); z still runs  */
   int32_t t_max;            /* horizon T_max (> 0)                                          */
   int32_t eos_token;        /* end-of-sequence id, or -1 for none                           */
@@ -95,7 +95,7 @@ typedef struct espo_params {
 typedef struct espo_state espo_state;
 
 /* Create the state for up to `capacity` trajectories over a vocabulary of V ids
- * (Algorithm 1, line 1: z = 0, t = 0, not done -- for every slot).
+ * (the initialisation of Algorithm 1: z = 0, t = 0, not done -- for every slot).
  *   out       host pointer that receives the handle
  *   seed      64-bit Philox key;  batch_id  rollout-batch number (< 2^30), part of the counter
  * Allocates device memory (this call and espo_free_state are the only ones that do for the
@@ -111,7 +111,7 @@ int espo_reset_state(espo_state* st, uint64_t batch_id, void* stream);
 /* Release the state and its device memory (synchronises the device). NULL is ignored. */
 void espo_free_state(espo_state* st);
 
-/* One decode step for n_rows trajectories (Algorithm 1, loop body; Eq. 5, 8, 9, 10).
+/* One decode step for n_rows trajectories (Algorithm 1, loop body; Eq. 6, 9, 10, 11).
  *   logits      device, [n_rows, V] row-major, element type logits_dtype, rows row_stride
  *               ELEMENTS apart (row_stride >= V).  Read exactly once from DRAM.  Entries may
  *               be -inf (masked ids).  The fast path needs a 16-byte aligned base and
@@ -143,7 +143,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride,
  * pointer may be NULL.  g, g_tilde and logp hold the values of each slot's latest step
  * (logp = log pi(a_t | s_t) under the temperature-scaled distribution).  t is the number
  * of tokens generated; t_stop is the index of the stop step or -1; sum_g, sum_g2 are the
- * double-precision sums over the slot's tokens that the batch statistics of Eq. 6-7 need. */
+ * double-precision sums over the slot's tokens that the batch statistics of Eq. 7-8 need. */
 int espo_state_view(espo_state* st, const float** z, const float** g, const float** g_tilde,
                     const float** logp, const int32_t** t, const uint8_t** status,
                     const int32_t** t_stop, const double** sum_g, const double** sum_g2);
@@ -163,8 +163,8 @@ int espo_compact_active(espo_state* st, int32_t* row_ids_out, int32_t* n_active_
 /* Copy the sticky device status word (ESPO_DEV_* bits) to *host_out.  Synchronises `stream`. */
 int espo_state_status(espo_state* st, uint32_t* host_out, void* stream);
 
-/* TD errors and GAE over B ragged trajectories (Eq. 3-4) with ESPO's failure transition
- * (Eq. 12).  Trajectory i owns tokens [off_i, off_i + lengths[i]) of the packed arrays,
+/* TD errors and GAE over B ragged trajectories (Eq. 4-5) with ESPO's failure transition
+ * (Eq. 13).  Trajectory i owns tokens [off_i, off_i + lengths[i]) of the packed arrays,
  * off = exclusive prefix sum of lengths.
  *   rewards, values  device float32 [total_tokens]
  *   lengths          device int32 [B] (>= 0; the stop-step token of a stopped trajectory is

@@ -1,7 +1,7 @@
 """ctypes loader for the ESPO reference oracle (``espo_oracle.cpp``).
 
 TEST INFRASTRUCTURE ONLY.  The oracle is a slow double-precision CPU statement of
-the method, written from the paper's equations (Sec. 3 Eq. 3-4, Sec. 4 Eq. 5-12,
+the method, written from the paper's equations (Sec. 3 Eq. 4-5, Sec. 4 Eq. 6-13,
 Algorithm 1).  Nothing in the product package imports this module; only the tests,
 the smoke check and the benchmark's CPU-baseline leg do.  It shares no code with
 the CUDA library.
@@ -41,7 +41,7 @@ def build(force: bool = False) -> str:
 
 
 class Params(C.Structure):
-    """Frozen per-batch parameters (Eq. 8-10, Algorithm 1 inputs)."""
+    """Frozen per-batch parameters (Eq. 9-11, Algorithm 1 inputs)."""
     _fields_ = [("temperature", C.c_double), ("mu_g", C.c_double), ("sigma2_g", C.c_double),
                 ("delta", C.c_double), ("clip_c", C.c_double), ("alpha_s", C.c_double),
                 ("beta", C.c_double), ("eps", C.c_double), ("warmup_complete", C.c_int32),
@@ -180,7 +180,7 @@ class Rollout:
 
 
 def advantages(rewards, values, lengths, stopped, gamma, lam, r_fail, direct=False) -> np.ndarray:
-    """GAE over packed ragged trajectories with the absorbing failure transition (Eq. 3-4, 12)."""
+    """GAE over packed ragged trajectories with the absorbing failure transition (Eq. 4-5, 13)."""
     r = np.ascontiguousarray(rewards, dtype=np.float64)
     v = np.ascontiguousarray(values, dtype=np.float64)
     L = np.ascontiguousarray(lengths, dtype=np.int32)

@@ -7,13 +7,13 @@
 // the same written definitions.
 //
 // What follows the paper, and where:
-//   * surrogate regret  g_t = max_a log pi(a|s_t) - log pi(a_t|s_t)   (Sec. 4.1, Eq. 5)
-//   * normalised signal g~_t = clip((g_t - mu_g)/sqrt(sigma_g^2 + delta), -c, c)  (Sec. 4.2, Eq. 8)
-//   * smoothed cumulative regret z_t = a_s z_{t-1} + (1-a_s) g~_t, z_0 = 0        (Sec. 4.2, Eq. 9)
-//   * value-gated stop  z_t > beta * max(V_phi(s_t), eps), only after warm-up     (Sec. 4.3, Eq. 10; Algorithm 1)
-//   * failure transition r_{T_stop} = r_fail, nothing bootstrapped past the end   (Sec. 4.4, Eq. 12)
+//   * surrogate regret  g_t = max_a log pi(a|s_t) - log pi(a_t|s_t)   (Sec. 4.1, Eq. 6)
+//   * normalised signal g~_t = clip((g_t - mu_g)/sqrt(sigma_g^2 + delta), -c, c)  (Sec. 4.2, Eq. 9)
+//   * smoothed cumulative regret z_t = a_s z_{t-1} + (1-a_s) g~_t, z_0 = 0        (Sec. 4.2, Eq. 10)
+//   * value-gated stop  z_t > beta * max(V_phi(s_t), eps), only after warm-up     (Sec. 4.3, Eq. 11; Algorithm 1)
+//   * failure transition r_{T_stop} = r_fail, nothing bootstrapped past the end   (Sec. 4.4, Eq. 13)
 //   * TD error and GAE  delta_t = r_t + gamma V(s_{t+1}) - V(s_t),
-//                       A_t = sum_l (gamma lambda)^l delta_{t+l}                  (Sec. 3, Eq. 3-4)
+//                       A_t = sum_l (gamma lambda)^l delta_{t+l}                  (Sec. 3, Eq. 4-5)
 //
 // What the paper leaves open and this file fixes (the same written convention the
 // CUDA library follows):
@@ -144,9 +144,9 @@ extern "C" {
 
 struct espo_oracle_params {
   double temperature;
-  double mu_g, sigma2_g, delta, clip_c;   // Eq. 8 (frozen for the whole rollout batch)
-  double alpha_s;                          // Eq. 9
-  double beta, eps;                        // Eq. 10
+  double mu_g, sigma2_g, delta, clip_c;   // Eq. 9 (frozen for the whole rollout batch)
+  double alpha_s;                          // Eq. 10
+  double beta, eps;                        // Eq. 11
   int32_t warmup_complete;                 // Algorithm 1: the test is gated, z is not
   int32_t t_max;                           // horizon T_max
   int32_t eos_token;                       // -1: none
@@ -157,7 +157,7 @@ enum { ORACLE_ACTIVE = 0, ORACLE_STOPPED = 1, ORACLE_EOS = 2, ORACLE_TMAX = 3, O
 
 struct espo_oracle_row_state {
   double z;          // smoothed cumulative regret
-  double sum_g;      // running sums over this trajectory's tokens (for the batch statistics of Eq. 6-7)
+  double sum_g;      // running sums over this trajectory's tokens (for the batch statistics of Eq. 7-8)
   double sum_g2;
   int64_t n_tokens;
   int32_t t;         // tokens generated so far
@@ -277,20 +277,20 @@ void espo_oracle_step_row(const double* logits, int64_t V, double value,
     if (ga <= gb && ga <= gj) out->runner_up = (int32_t)ra.runner;
   }
 
-  // Eq. 5: the normaliser cancels in the difference of the two log-probabilities.
+  // Eq. 6: the normaliser cancels in the difference of the two log-probabilities.
   const double x_tok = x[token];
   const double g = greedy ? 0.0 : (m - x_tok);
   const double logp = greedy ? 0.0 : (x_tok - m - out->log_s);
 
-  // Eq. 8 with the frozen batch statistics.
+  // Eq. 9 with the frozen batch statistics.
   double gt = (g - p->mu_g) / std::sqrt(p->sigma2_g + p->delta);
   if (gt > p->clip_c) gt = p->clip_c;
   if (gt < -p->clip_c) gt = -p->clip_c;
 
-  // Eq. 9: updated on every step, warm-up or not (Algorithm 1 updates z before the gated test).
+  // Eq. 10: updated on every step, warm-up or not (Algorithm 1 updates z before the gated test).
   const double z = p->alpha_s * st->z + (1.0 - p->alpha_s) * gt;
 
-  // Eq. 10, strict inequality; a NaN value estimate never stops.
+  // Eq. 11, strict inequality; a NaN value estimate never stops.
   const double thr = p->beta * std::fmax(value, p->eps);
   const bool fires = (p->warmup_complete != 0) && !std::isnan(value) && (z > thr);
 
@@ -376,15 +376,15 @@ void espo_oracle_step_batch_f32(const float* logits, int64_t V, const double* va
 }
 
 // ---------------------------------------------------------------------------
-// Advantages over ragged, truncated trajectories (Eq. 3-4 with the failure
-// transition of Eq. 12).  Trajectory i owns tokens [off_i, off_i + L_i) of the
+// Advantages over ragged, truncated trajectories (Eq. 4-5 with the failure
+// transition of Eq. 13).  Trajectory i owns tokens [off_i, off_i + L_i) of the
 // packed arrays, off = exclusive prefix sum of lengths.
 //   r'_t = rewards[t], except r'_{L-1} = r_fail when stopped[i] (replaces, not adds)
 //   V_L := 0 for every trajectory: nothing is bootstrapped past its last token
 //   delta_t = r'_t + gamma V_{t+1} - V_t
 // ---------------------------------------------------------------------------
 
-// Literal Eq. 4: A_t = sum_{l=0}^{L-1-t} (gamma*lambda)^l delta_{t+l}.  O(L^2).
+// Literal Eq. 5: A_t = sum_{l=0}^{L-1-t} (gamma*lambda)^l delta_{t+l}.  O(L^2).
 void espo_oracle_advantages_direct(const double* rewards, const double* values,
                                    const int32_t* lengths, const uint8_t* stopped, int32_t B,
                                    double gamma, double lambda, double r_fail, double* adv_out) {

@@ -33,7 +33,7 @@ class EspoError(RuntimeError):
 
 
 class espo_params(C.Structure):
-    """Mirror of the C struct: parameters frozen for a rollout batch (Eq. 8-10, Algorithm 1)."""
+    """Mirror of the C struct: parameters frozen for a rollout batch (Eq. 9-11, Algorithm 1)."""
     _fields_ = [("temperature", C.c_float), ("mu_g", C.c_float), ("sigma2_g", C.c_float),
                 ("delta", C.c_float), ("clip_c", C.c_float), ("alpha_s", C.c_float),
                 ("beta", C.c_float), ("eps", C.c_float), ("warmup_complete", C.c_int32),
@@ -213,7 +213,7 @@ def espo_state_status(state: EspoState, stream=None) -> int:
 def espo_advantages(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.Tensor, stopped: torch.Tensor,
                     gamma: float, lam: float, r_fail: float, adv_out: torch.Tensor,
                     total_tokens: Optional[int] = None, stream=None) -> None:
-    """TD + GAE over packed ragged trajectories with the failure transition (Eq. 3-4, 12); see ``espo.h``."""
+    """TD + GAE over packed ragged trajectories with the failure transition (Eq. 4-5, 13); see ``espo.h``."""
     for t, n, dt in ((rewards, "rewards", torch.float32), (values, "values", torch.float32),
                      (adv_out, "adv_out", torch.float32), (lengths, "lengths", torch.int32),
                      (stopped, "stopped", torch.uint8)):

@@ -1,5 +1,5 @@
-// TD errors and GAE over ragged, truncated trajectories (Eq. 3-4) with ESPO's absorbing
-// failure transition (Eq. 12), for sm_100a.
+// TD errors and GAE over ragged, truncated trajectories (Eq. 4-5) with ESPO's absorbing
+// failure transition (Eq. 13), for sm_100a.
 //
 // The packed token array is cut into fixed chunks of kAdvChunk tokens regardless of where
 // trajectories begin and end, so every CTA moves the same number of bytes (12 per token:

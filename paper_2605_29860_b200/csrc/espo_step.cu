@@ -2,8 +2,8 @@
 //
 // One launch performs, for every logit row of the batch, the body of the rollout loop
 // (Algorithm 1): log-softmax statistics, Gumbel-max sampling, the surrogate regret of
-// Eq. 5, its normalisation (Eq. 8) and smoothing (Eq. 9), the value-gated stop test
-// (Eq. 10) and the per-trajectory bookkeeping.
+// Eq. 6, its normalisation (Eq. 9) and smoothing (Eq. 10), the value-gated stop test
+// (Eq. 11) and the per-trajectory bookkeeping.
 //
 // Shape of the kernel
 //   * The [n_rows, V] logits are a sequence of n_rows * ceil(V/1024) blocks of 1024 ids.  A
@@ -21,7 +21,7 @@
 //     blocks, the streaming warps) take rows from the queue, add the CTA's share to the
 //     row's ticket in global memory, and whoever completes the ticket merges the block
 //     records in a fixed order (so results do not depend on the grid), draws the token,
-//     applies Eq. 5, 8, 9, 10 and writes the outputs and the trajectory state.
+//     applies Eq. 6, 9, 10, 11 and writes the outputs and the trajectory state.
 //   * A CTA walks its range starting with the row it shares with the next CTA, then the row it
 //     shares with the previous one, then its whole rows: shared rows complete early in the
 //     launch instead of all at its end.
@@ -40,7 +40,7 @@
 namespace espo {
 
 constexpr int kMaxStepThreads = 1024;
-constexpr int kMaxConsumerWarps = kMaxStepThreads / 32 - 1;   // one more warp is the finalizer
+constexpr int kMaxConsumerWarps = kMaxStepThreads / 32 - 1;   // at least one more warp is a finalizer
 constexpr int kMaxQueue = 4096;
 
 struct StepArgs {
@@ -54,7 +54,7 @@ struct StepArgs {
   // tiling
   int nblk;                 // 1024-id blocks per row
   long long total_blocks;   // n_rows * nblk
-  int warps, stages, stage_bytes, queue_cap;
+  int warps, fin_warps, stages, stage_bytes, queue_cap;   // streaming warps, finalizer warps, ring depth
   int local_rows;           // rows whose block records fit in the CTA's shared-memory table (0: none)
   int noise_rows;           // rows whose block-level noise fits in the CTA's shared-memory table
   // trajectory state (indexed by slot)
@@ -434,7 +434,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
   }
 
   if (lane == 0) {
-    // Eq. 5: the normaliser cancels; Eq. 8; Eq. 9; Eq. 10.
+    // Eq. 6: the normaliser cancels; Eq. 9; Eq. 10; Eq. 11.
     const float g = a.greedy ? 0.f : (M - l_tok) * a.inv_temp;
     const float logp = a.greedy ? 0.f : (-g - log_S);
     float gt = (g - a.mu_g) * a.inv_sigma;
@@ -558,8 +558,8 @@ __device__ void drain_queue(const StepArgs& a, const CtaRange& cr, StepCtrl* ctr
 // The finalizer warp's first job, while the streaming warps fetch their first blocks: read the
 // state of every row the range touches and draw the block-level noise of those rows.
 template <int SAMPLER>
-__device__ void prepare_rows(const StepArgs& a, const CtaRange& cr, const RowTables& tb, int lane) {
-  for (int k = 0; k < cr.n_local; ++k) {
+__device__ void prepare_rows(const StepArgs& a, const CtaRange& cr, const RowTables& tb, int lane, int first, int step) {
+  for (int k = first; k < cr.n_local; k += step) {
     const int row = (int)(cr.r_first + k);
     const RowPre pre = prefetch_row(a, row);
     if (lane == 0) tb.pre[k] = pre;
@@ -772,9 +772,9 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
     }
   }
   // The finalizer warp comes here at once; streaming warps join when they run out of blocks.
-  if (warp == W) {
+  if (warp >= W) {
     cta_rendezvous(blockDim.x);   // (A)
-    prepare_rows<SAMPLER>(a, cr, tb, lane);
+    prepare_rows<SAMPLER>(a, cr, tb, lane, warp - W, a.fin_warps);   // the finalizer warps share the rows
   }
   drain_queue<ES, SAMPLER>(a, cr, ctrl, tb, lane);
 }
@@ -960,9 +960,16 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   a.stage_bytes = kBlockIds * es;
   // Launch shape: ctas_per_sm CTAs of `warps` streaming warps (+1 finalizer warp), `stages` blocks in flight per warp.
   int ctas_per_sm = st->cfg_ctas_per_sm ? st->cfg_ctas_per_sm : 1;
+  // Finalizer warps per CTA: one row takes a warp about 5 us to finalize, and an SM streams a row in
+  // row_bytes / ~43 GB/s; short rows need several finalizers to keep up with the streaming warps.
+  const double row_us = (double)st->V * es / 43e3;
+  int fin = (int)ceil(5.0 / (row_us * ctas_per_sm));
+  fin = fin < 1 ? 1 : (fin > 8 ? 8 : fin);
+  const int max_warps = (kMaxStepThreads / 32 < 64 / ctas_per_sm) ? kMaxStepThreads / 32 : 64 / ctas_per_sm;
   int warps = st->cfg_warps ? st->cfg_warps : (es == 2 ? 31 : 15);
   int stages = st->cfg_stages ? st->cfg_stages : 2;
-  if ((warps + 1) * 32 * ctas_per_sm > 2048) warps = 2048 / (32 * ctas_per_sm) - 1;
+  if (warps + fin > max_warps) warps = max_warps - fin;
+  if (warps < 1) { warps = 1; fin = (fin < max_warps - 1) ? fin : (max_warps - 1 < 1 ? 1 : max_warps - 1); }
   long long grid = (long long)st->sm_count * ctas_per_sm;
   if (grid > a.total_blocks) grid = a.total_blocks;
   const long long blocks_per_cta = (a.total_blocks + grid - 1) / grid;
@@ -988,6 +995,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   const long long per_warp = (blocks_per_cta + warps - 1) / warps;
   if (per_warp < stages) stages = (int)per_warp;
   a.warps = warps;
+  a.fin_warps = fin;
   a.stages = stages;
   const size_t smem = footprint(warps, stages);
   if (smem > (size_t)st->max_smem) return ESPO_ERR_CAPACITY;
@@ -1014,7 +1022,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
 
   const bool bulk = ((uintptr_t)logits % 16 == 0) && (a.row_stride_bytes % 16 == 0) && (((size_t)st->V * es) % 16 == 0);
   StepKernel k = pick_kernel(es, p->sampler, bulk);
-  k<<<(unsigned)grid, (unsigned)(warps + 1) * 32u, smem, (cudaStream_t)stream>>>(a);
+  k<<<(unsigned)grid, (unsigned)(warps + fin) * 32u, smem, (cudaStream_t)stream>>>(a);
   ESPO_CUDA_TRY(cudaGetLastError());
   return ESPO_OK;
 }

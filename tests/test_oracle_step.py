@@ -38,7 +38,7 @@ def test_log_softmax_matches_library_and_normalises(temperature):
 
 
 def test_step_reports_the_log_prob_and_gap_of_its_token():
-    # Eq. 5 the long way: two normalised log-probabilities, subtracted.
+    # Eq. 6 the long way: two normalised log-probabilities, subtracted.
     rng = _rng(2)
     V = 3000
     x = _peaked_logits(rng, 6, V)
@@ -209,7 +209,7 @@ def test_unusable_rows_are_flagged_not_sampled():
         assert ro.states[0].status == oracle.BAD and ro.states[0].t == 0 and ro.states[0].z == 0.0
 
 
-# --------------------------------------------------------------------------- Eq. 8-10
+# --------------------------------------------------------------------------- Eq. 9-11
 
 
 def _forced(ro, x, v, p, tok):
