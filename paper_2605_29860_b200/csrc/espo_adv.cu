@@ -2,17 +2,19 @@
 // failure transition (Eq. 13), for sm_100a.
 //
 // The packed token array is cut into fixed chunks of kAdvChunk tokens regardless of where
-// trajectories begin and end, so every CTA moves the same number of bytes (12 per token:
-// reward and value in, advantage out) whatever the length mix is.  Within a chunk the
-// backward recursion A_t = delta_t + k_t A_{t+1} (k_t = gamma*lambda, or 0 on a trajectory's
-// last token) is a scan over affine maps X -> b + a X: each thread composes the maps of its
-// 8 tokens, a warp-shuffle suffix scan and a small cross-warp pass compose them across the
-// CTA.  A chunk whose last token is not a trajectory end needs A of the next chunk's first
-// token; chunks are handed out from the END of the array by an atomic counter and pass that
-// value backwards through per-chunk descriptors (aggregate map first, final value when
-// known), so the array is read and written exactly once.  The maps are composed in double
-// precision, which costs nothing next to the memory traffic and keeps gamma*lambda = 1 sums
-// over 16k tokens exact to float32 rounding of the result.
+// trajectories begin and end, and every CTA of a persistent grid takes an equal, contiguous
+// range of chunks, so every CTA moves the same number of bytes (12 per token: reward and
+// value in, advantage out) whatever the length mix is.  Within a chunk the backward recursion
+// A_t = delta_t + k_t A_{t+1} (k_t = gamma*lambda, or 0 on a trajectory's last token) is a scan
+// over affine maps X -> b + a X: a thread folds its 16 consecutive tokens, the 256 threads'
+// maps are composed by a warp-shuffle suffix scan and a small cross-warp pass, all in double
+// precision (with gamma*lambda = 1 an advantage is a sum of up to 16k TD errors).  A CTA walks
+// its range from the highest chunk down and carries the value that follows a chunk in shared
+// memory.  The value that follows its highest chunk belongs to a trajectory that continues
+// in the next CTA's range: the CTA obtains it by folding (reading only) the rest of that one
+// trajectory first -- at most one trajectory's worth of extra reads per CTA, usually served by
+// L2 -- so CTAs never wait for one another.  Chunks reach shared memory through a two-stage
+// ring of bulk asynchronous copies (TMA without a tensor map) issued two chunks ahead.
 //
 // A small preparation kernel turns lengths into offsets and tells every chunk which
 // trajectory its first token belongs to.
@@ -29,18 +31,16 @@
 namespace espo {
 
 constexpr int kAdvThreads = 256;
-constexpr int kAdvPerThread = 8;
-constexpr int kAdvChunk = kAdvThreads * kAdvPerThread;   // 2048 tokens
+constexpr int kAdvPerThread = 16;
+constexpr int kAdvChunk = kAdvThreads * kAdvPerThread;   // 4096 tokens
 constexpr int kAdvWarps = kAdvThreads / 32;
+constexpr int kAdvCtasPerSm = 3;
+constexpr int kMaxDevicesAdv = 64;
 constexpr int kPrepThreads = 1024;
 
 struct AdvWorkspace {
   long long* offsets;     // [B+1] exclusive prefix sum of lengths
   int* chunk_first;       // [nchunks] trajectory that owns the chunk's first token
-  unsigned* flag;         // [nchunks] epoch*4 + {1: aggregate published, 2: final value published}
-  double2* agg;           // [nchunks] chunk map X -> agg.y + agg.x * X
-  double* fin;            // [nchunks] A of the chunk's first token
-  unsigned* counters;     // [0] next chunk ticket, [1] chunks finished
   unsigned* status;       // sticky ESPO_DEV_* bits
 };
 
@@ -55,7 +55,6 @@ struct AdvArgs {
   int nchunks;
   double gamma, gl;       // gamma, gamma*lambda
   float r_fail;
-  unsigned epoch4;        // epoch * 4
   AdvWorkspace ws;
 };
 
@@ -117,188 +116,245 @@ struct Map {   // X -> b + a * X
 __device__ __forceinline__ Map compose(const Map& lo, const Map& hi) { return Map{lo.a * hi.a, fma(lo.a, hi.b, lo.b)}; }
 
 __device__ __forceinline__ double shfl_down_d(double v, int o) { return __shfl_down_sync(kFullMask, v, o); }
+__device__ __forceinline__ double shfl_up_d(double v, int o) { return __shfl_up_sync(kFullMask, v, o); }
+__device__ __forceinline__ double shfl_d(double v, int src) { return __shfl_sync(kFullMask, v, src); }
 
-__global__ void __launch_bounds__(kAdvThreads) espo_adv_scan_kernel(const AdvArgs a) {
-  __shared__ __align__(16) unsigned char flags[kAdvChunk];   // bit0: last token of a trajectory, bit1: it was stopped
+// Shared memory of the scan kernel: two stages, each one chunk of rewards, one chunk of values followed by the
+// value of the token after the chunk, and one flag byte per token.
+constexpr int kAdvVStride = kAdvChunk + 4;      // floats; keeps the second stage 16-byte aligned
+constexpr size_t kAdvSmemBytes = 2 * sizeof(float) * kAdvChunk + 2 * sizeof(float) * kAdvVStride + 2 * kAdvChunk + 2 * sizeof(uint64_t);
+
+__global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kernel(const AdvArgs a) {
+  extern __shared__ __align__(128) unsigned char adv_smem[];
+  float* rbuf = reinterpret_cast<float*>(adv_smem);
+  float* vbuf = rbuf + 2 * kAdvChunk;
+  unsigned char* flagbuf = reinterpret_cast<unsigned char*>(vbuf + 2 * kAdvVStride);   // bit0: last token of a trajectory, bit1: it was stopped
+  uint64_t* mbar = reinterpret_cast<uint64_t*>(flagbuf + 2 * kAdvChunk);
   __shared__ Map warp_agg[kAdvWarps];
-  __shared__ float warp_first_v[kAdvWarps];
-  __shared__ int chunk_s;
-  __shared__ double carry_s;
+  __shared__ double pw[kAdvPerThread + 1];                   // (gamma*lambda)^i
+  __shared__ double carry_buf[2];                            // value that follows the chunk held by each stage
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) chunk_s = a.nchunks - 1 - (int)atomicAdd(a.ws.counters, 1u);   // highest positions first
-  reinterpret_cast<unsigned long long*>(flags)[tid] = 0ull;
-  __syncthreads();
-  const int j = chunk_s;
-  const long long p0 = (long long)j * kAdvChunk;
-  const int n = (int)min((long long)kAdvChunk, a.total - p0);
+  const double r_fail_d = (double)a.r_fail;
   const int q0 = tid * kAdvPerThread;
 
-  // ---- this thread's 8 rewards and values (issued before anything that depends on the prep data) ----
-  float r[kAdvPerThread], v[kAdvPerThread + 1];
+  // this CTA's chunks: [c_lo, c_hi), walked from c_hi - 1 down
+  const int c_lo = (int)((long long)blockIdx.x * a.nchunks / gridDim.x);
+  const int c_hi = (int)((long long)(blockIdx.x + 1) * a.nchunks / gridDim.x);
+
+  // Marks the trajectory ends that fall into chunk `jj` in the flag bytes of `stage`.  The three loads of a
+  // trajectory are independent of one another.
+  auto mark_ends = [&](int jj, int stage) {
+    unsigned char* fl = flagbuf + stage * kAdvChunk;
+    const long long p0 = (long long)jj * kAdvChunk;
+    const long long p_end = min(p0 + kAdvChunk, a.total);
+    for (int i = __ldg(a.ws.chunk_first + jj) + tid; i < a.B; i += kAdvThreads) {
+      const long long o0 = __ldcg(a.ws.offsets + i);
+      const long long o1 = __ldcg(a.ws.offsets + i + 1);
+      const unsigned st = a.stopped[i];
+      if (o0 >= p_end) break;
+      if (o1 > o0 && o1 - 1 >= p0 && o1 - 1 < p_end) fl[o1 - 1 - p0] = (unsigned char)(1u | (st ? 2u : 0u));
+    }
+  };
+
+  // Starts the copy of chunk `jj` into `stage`; called by every thread.  A full chunk is two bulk copies
+  // (plus 16 bytes for the value after the chunk) that complete on the stage's mbarrier; the array's ragged
+  // last chunk is copied with ordinary loads and the barrier completed by hand.
+  auto fetch = [&](int jj, int stage) {
+    const long long p0 = (long long)jj * kAdvChunk;
+    float* rs = rbuf + stage * kAdvChunk;
+    float* vs = vbuf + stage * kAdvVStride;
+    if (p0 + kAdvChunk <= a.total) {
+      if (tid == 0) {
+        const bool tail16 = (p0 + kAdvChunk + 4 <= a.total);      // the 16 bytes after the chunk exist
+        fence_proxy_async();                                       // earlier reads of the stage come first
+        mbar_arrive_expect_tx(&mbar[stage], 2u * sizeof(float) * kAdvChunk + (tail16 ? 16u : 0u));
+        bulk_copy_g2s(rs, a.rewards + p0, sizeof(float) * kAdvChunk, &mbar[stage]);
+        bulk_copy_g2s(vs, a.values + p0, sizeof(float) * kAdvChunk, &mbar[stage]);
+        if (tail16) bulk_copy_g2s(vs + kAdvChunk, a.values + p0 + kAdvChunk, 16u, &mbar[stage]);
+        else vs[kAdvChunk] = (p0 + kAdvChunk < a.total) ? __ldg(a.values + p0 + kAdvChunk) : 0.f;
+      }
+    } else {
+      const int n = (int)(a.total - p0);
+      for (int q = tid; q < kAdvChunk; q += kAdvThreads) {
+        rs[q] = (q < n) ? __ldcs(a.rewards + p0 + q) : 0.f;
+        vs[q] = (q < n) ? __ldcs(a.values + p0 + q) : 0.f;
+      }
+      if (tid == 0) vs[kAdvChunk] = 0.f;
+      __syncthreads();
+      if (tid == 0) mbar_arrive(&mbar[stage]);
+    }
+  };
+
+  uint32_t phase[2] = {0u, 0u};
+  unsigned last_mask = 0;
+  double d[kAdvPerThread];
+  Map m, after;
+
+  // Waits for `stage`, folds the chunk `jj` it holds: leaves the thread's TD errors in d[], its end mask in
+  // last_mask, its own map in m and the map of everything after the thread inside the chunk in `after`; the
+  // stage's flag bytes are cleared for their next use.  Contains one __syncthreads().
+  auto fold = [&](int jj, int stage) {
+    const float* rs = rbuf + stage * kAdvChunk;
+    const float* vs = vbuf + stage * kAdvVStride;
+    const long long p0 = (long long)jj * kAdvChunk;
+    if (!mbar_wait_bounded(&mbar[stage], phase[stage], nullptr)) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
+    phase[stage] ^= 1u;
+    float r[kAdvPerThread], v[kAdvPerThread];
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const int q = q0 + 4 * h;
-    if (q + 4 <= n) {
-      const float4 rr = __ldcs(reinterpret_cast<const float4*>(a.rewards + p0 + q));
-      const float4 vv = __ldcs(reinterpret_cast<const float4*>(a.values + p0 + q));
+    for (int h = 0; h < kAdvPerThread / 4; ++h) {
+      const float4 rr = *reinterpret_cast<const float4*>(rs + q0 + 4 * h);
+      const float4 vv = *reinterpret_cast<const float4*>(vs + q0 + 4 * h);
       r[4 * h] = rr.x; r[4 * h + 1] = rr.y; r[4 * h + 2] = rr.z; r[4 * h + 3] = rr.w;
       v[4 * h] = vv.x; v[4 * h + 1] = vv.y; v[4 * h + 2] = vv.z; v[4 * h + 3] = vv.w;
-    } else {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        r[4 * h + e] = (q + e < n) ? __ldcs(a.rewards + p0 + q + e) : 0.f;
-        v[4 * h + e] = (q + e < n) ? __ldcs(a.values + p0 + q + e) : 0.f;
-      }
     }
-  }
-  // value of the token after this thread's last one: next lane, next warp, or next chunk
-  float v_after = __shfl_down_sync(kFullMask, v[0], 1);
-  if (lane == 0) warp_first_v[warp] = v[0];
+    const float v_after = vs[q0 + kAdvPerThread];   // the next thread's first value; for the last thread, the next chunk's
+    uint4* fp = reinterpret_cast<uint4*>(flagbuf + stage * kAdvChunk) + tid;
+    const uint4 f16 = *fp;
+    *fp = make_uint4(0u, 0u, 0u, 0u);
+    const unsigned fw[4] = {f16.x, f16.y, f16.z, f16.w};
+    unsigned fail_mask = 0;
+    last_mask = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {   // gather bit 0 (resp. bit 1) of four bytes into four adjacent bits
+      last_mask |= (((fw[w] & 0x01010101u) * 0x01020408u) >> 24) << (4 * w);
+      fail_mask |= ((((fw[w] >> 1) & 0x01010101u) * 0x01020408u) >> 24) << (4 * w);
+    }
+    {
+      // the array's very last token ends a trajectory even if the lengths are inconsistent
+      const long long e_last = a.total - 1 - p0 - q0;
+      if (e_last >= 0 && e_last < kAdvPerThread) last_mask |= 1u << (int)e_last;
+    }
+    fail_mask &= last_mask;
+    double mb = 0.0;
+    double vd_next = (double)v_after;
+#pragma unroll
+    for (int e = kAdvPerThread - 1; e >= 0; --e) {
+      const bool last = (last_mask >> e) & 1u;
+      const double vd = (double)v[e];
+      const double rd = ((fail_mask >> e) & 1u) ? r_fail_d : (double)r[e];
+      const double de = (last ? rd : fma(a.gamma, vd_next, rd)) - vd;
+      d[e] = de;
+      mb = last ? de : fma(a.gl, mb, de);
+      vd_next = vd;
+    }
+    // Tokens past the end of the array (only in its last chunk) read as zeros; the array's last token is a
+    // forced trajectory end, so nothing of them reaches a stored result.
+    m = Map{last_mask ? 0.0 : pw[kAdvPerThread], mb};   // X survives the thread only if no trajectory ends in it
+    Map inc = m;   // inclusive suffix inside the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      Map hi{shfl_down_d(inc.a, o), shfl_down_d(inc.b, o)};
+      if (lane + o < 32) inc = compose(inc, hi);
+    }
+    if (lane == 0) warp_agg[warp] = inc;
+    after = Map{shfl_down_d(inc.a, 1), shfl_down_d(inc.b, 1)};   // exclusive within the warp
+    if (lane == 31) after = Map{1.0, 0.0};
+    __syncthreads();   // warp aggregates written; every thread has read its part of the stage
+    for (int w = warp + 1; w < kAdvWarps; ++w) after = compose(after, warp_agg[w]);
+  };
 
-  // ---- mark trajectory ends inside the chunk ----
+  if (tid == 0) {
+    mbar_init(&mbar[0], 1);
+    mbar_init(&mbar[1], 1);
+    mbar_init_fence();
+    double p = 1.0;
+    for (int i = 0; i <= kAdvPerThread; ++i) { pw[i] = p; p *= a.gl; }
+  }
+  reinterpret_cast<uint4*>(flagbuf)[tid] = make_uint4(0u, 0u, 0u, 0u);
+  reinterpret_cast<uint4*>(flagbuf)[tid + kAdvThreads] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  if (c_lo >= c_hi) return;
+
+  // ---- the value that follows the CTA's highest chunk: fold the rest of the trajectory that crosses the range's
+  //      upper end (chunks c_hi, c_hi + 1, ... up to the first one that holds a trajectory end).  Stage 1 meanwhile
+  //      receives the highest chunk of the range. ----
+  fetch(c_hi - 1, 1);
+  mark_ends(c_hi - 1, 1);
+  double carry = 0.0;
   {
-    const long long p_end = p0 + n;
-    for (int i = a.ws.chunk_first[j] + tid; i < a.B; i += kAdvThreads) {
-      const long long o0 = a.ws.offsets[i];
-      if (o0 >= p_end) break;
-      const long long o1 = a.ws.offsets[i + 1];
-      if (o1 > o0 && o1 - 1 >= p0 && o1 - 1 < p_end) flags[o1 - 1 - p0] = (unsigned char)(1u | (a.stopped[i] ? 2u : 0u));
+    Map acc{1.0, 0.0};
+    for (int jh = c_hi; jh < a.nchunks && acc.a != 0.0; ++jh) {
+      fetch(jh, 0);
+      mark_ends(jh, 0);
+      __syncthreads();            // flags marked
+      fold(jh, 0);
+      const Map whole = compose(m, after);                      // thread 0: the whole chunk
+      const double wa = __shfl_sync(kFullMask, whole.a, 0), wb = __shfl_sync(kFullMask, whole.b, 0);
+      if (tid == 0) { carry_buf[0] = wa; carry_buf[1] = wb; }
+      __syncthreads();
+      acc = compose(acc, Map{carry_buf[0], carry_buf[1]});
+      __syncthreads();            // carry_buf free again
     }
+    carry = acc.b;                // past the end of the array the value is 0
   }
+  if (tid == 0) carry_buf[1] = carry;
+
+  // ---- the range, from its highest chunk down; chunk j sits in stage (c_hi - 1 - j + 1) & 1 ----
+  if (c_hi - 2 >= c_lo) { fetch(c_hi - 2, 0); mark_ends(c_hi - 2, 0); }
   __syncthreads();
-  if (lane == 31) {
-    if (warp + 1 < kAdvWarps) v_after = warp_first_v[warp + 1];
-    else v_after = (p0 + kAdvChunk < a.total) ? __ldg(a.values + p0 + kAdvChunk) : 0.f;
-  }
-  v[kAdvPerThread] = v_after;
+  int s = 1;
+  for (int j = c_hi - 1; j >= c_lo; --j, s ^= 1) {
+    const long long p0 = (long long)j * kAdvChunk;
+    const int n = (int)min((long long)kAdvChunk, a.total - p0);
+    int n_in = n - q0;       // tokens of this thread that exist
+    n_in = n_in < 0 ? 0 : (n_in > kAdvPerThread ? kAdvPerThread : n_in);
+    fold(j, s);
+    const double carry_in = carry_buf[s];
+    if (tid == 0) {
+      const Map whole = compose(m, after);
+      carry_buf[s ^ 1] = fma(whole.a, carry_in, whole.b);       // what follows the next (lower) chunk
+    }
+    // the stage is free: start the copy of the chunk two below, and mark its trajectory ends
+    if (j - 2 >= c_lo) { fetch(j - 2, s); mark_ends(j - 2, s); }
 
-  // ---- per-token TD error and coefficient; compose the thread's map right to left ----
-  const unsigned long long f8 = reinterpret_cast<const unsigned long long*>(flags)[tid];
-  double delta[kAdvPerThread];
-  unsigned last_mask = 0;
-  Map m{1.0, 0.0};
+    // ---- replay the thread's tokens with the value that follows them ----
+    double x = fma(after.a, carry_in, after.b);
+    float out[kAdvPerThread];
 #pragma unroll
-  for (int e = kAdvPerThread - 1; e >= 0; --e) {
-    const unsigned f = (unsigned)(f8 >> (8 * e)) & 0xffu;
-    const bool in = (q0 + e < n);
-    // the array's very last token ends a trajectory even if the lengths are inconsistent
-    const bool last = (f & 1u) || (p0 + q0 + e == a.total - 1);
-    const double rew = (last && (f & 2u)) ? (double)a.r_fail : (double)r[e];
-    const double d = rew + (last ? 0.0 : a.gamma * (double)v[e + 1]) - (double)v[e];
-    delta[e] = d;
-    if (last) last_mask |= 1u << e;
-    if (in) {
-      const double k = last ? 0.0 : a.gl;
-      m = Map{k * m.a, fma(k, m.b, d)};
-    }
-  }
-
-  // ---- suffix scan over the CTA: what comes after each thread, as a map of the chunk's carry-in ----
-  Map inc = m;   // inclusive: this thread and everything after it inside the warp
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    Map hi{shfl_down_d(inc.a, o), shfl_down_d(inc.b, o)};
-    if (lane + o < 32) inc = compose(inc, hi);
-  }
-  if (lane == 0) warp_agg[warp] = inc;
-  Map after{shfl_down_d(inc.a, 1), shfl_down_d(inc.b, 1)};   // exclusive within the warp
-  if (lane == 31) after = Map{1.0, 0.0};
-  __syncthreads();
-  for (int w = warp + 1; w < kAdvWarps; ++w) after = compose(after, warp_agg[w]);
-
-  // ---- chunk descriptor and carry-in ----
-  if (tid == 0) {
-    const Map whole = compose(m, after);     // the whole chunk
-    const bool has_next = (p0 + kAdvChunk < a.total);
-    // Tokens after the chunk's last trajectory end still need the value that follows the chunk,
-    // even though the chunk as a whole (whole.a == 0) passes nothing through.
-    const bool need_carry = has_next && !(flags[n - 1] & 1u);
-    volatile unsigned* my_flag = reinterpret_cast<volatile unsigned*>(a.ws.flag + j);
-    if (whole.a == 0.0) {                    // A of the first token does not depend on what follows
-      a.ws.fin[j] = whole.b;
-      __threadfence();
-      *my_flag = a.epoch4 | 2u;
-    } else {
-      a.ws.agg[j] = make_double2(whole.a, whole.b);
-      __threadfence();
-      *my_flag = a.epoch4 | 1u;
-    }
-    double carry = 0.0;
-    if (need_carry) {
-      // walk forward through the chunks after this one until the chain closes
-      Map acc{1.0, 0.0};
-      int jj = j + 1;
-      bool resolved = false;
-      for (uint32_t it = 0; it < kPollSpinLimit && !resolved; ++it) {
-        const unsigned f = *reinterpret_cast<volatile unsigned*>(a.ws.flag + jj);
-        if (f == (a.epoch4 | 2u)) {
-          __threadfence();
-          carry = fma(acc.a, __ldcg(a.ws.fin + jj), acc.b);
-          resolved = true;
-        } else if (f == (a.epoch4 | 1u)) {
-          __threadfence();
-          const double2 g = __ldcg(a.ws.agg + jj);
-          acc = compose(acc, Map{g.x, g.y});
-          ++jj;
-          if (acc.a == 0.0 || jj >= a.nchunks) { carry = acc.b; resolved = true; }
-        } else {
-          __nanosleep(40);
-        }
-      }
-      if (!resolved) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
-    }
-    if (whole.a != 0.0) {
-      a.ws.fin[j] = fma(whole.a, carry, whole.b);
-      __threadfence();
-      *my_flag = a.epoch4 | 2u;
-    }
-    carry_s = carry;
-  }
-  __syncthreads();
-
-  // ---- replay the thread's tokens with the now known value that follows them ----
-  double x = fma(after.a, carry_s, after.b);
-  float out[kAdvPerThread];
-#pragma unroll
-  for (int e = kAdvPerThread - 1; e >= 0; --e) {
-    if (q0 + e < n) {
-      const double k = ((last_mask >> e) & 1u) ? 0.0 : a.gl;
-      x = fma(k, x, delta[e]);
+    for (int e = kAdvPerThread - 1; e >= 0; --e) {
+      x = ((last_mask >> e) & 1u) ? d[e] : fma(a.gl, x, d[e]);
       out[e] = (float)x;
-    } else {
-      out[e] = 0.f;
     }
-  }
+    if (n_in == kAdvPerThread) {
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const int q = q0 + 4 * h;
-    if (q + 4 <= n) {
-      __stcs(reinterpret_cast<float4*>(a.adv + p0 + q), make_float4(out[4 * h], out[4 * h + 1], out[4 * h + 2], out[4 * h + 3]));
+      for (int h = 0; h < kAdvPerThread / 4; ++h)
+        __stcs(reinterpret_cast<float4*>(a.adv + p0 + q0) + h, make_float4(out[4 * h], out[4 * h + 1], out[4 * h + 2], out[4 * h + 3]));
     } else {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) if (q + e < n) a.adv[p0 + q + e] = out[4 * h + e];
+      for (int e = 0; e < kAdvPerThread; ++e) if (e < n_in) a.adv[p0 + q0 + e] = out[e];
     }
+    __syncthreads();   // the next chunk's flags and carry are in place
   }
+}
 
-  // ---- the last CTA to finish rewinds the counters for the next call ----
-  if (tid == 0) {
-    __threadfence();
-    if (atomicAdd(a.ws.counters + 1, 1u) == (unsigned)a.nchunks - 1u) {
-      a.ws.counters[0] = 0u;
-      a.ws.counters[1] = 0u;
-    }
+// Launches both kernels; `sm_count` sizes the persistent grid of the scan.
+static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
+  static bool attr_set[kMaxDevicesAdv] = {};
+  int dev = 0;
+  ESPO_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < kMaxDevicesAdv && !attr_set[dev]) {
+    ESPO_CUDA_TRY(cudaFuncSetAttribute((const void*)espo_adv_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kAdvSmemBytes));
+    attr_set[dev] = true;
   }
+  espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
+  ESPO_CUDA_TRY(cudaGetLastError());
+  long long grid = (long long)sm_count * kAdvCtasPerSm;
+  if (grid > a.nchunks) grid = a.nchunks;
+  espo_adv_scan_kernel<<<(unsigned)grid, kAdvThreads, kAdvSmemBytes, s>>>(a);
+  ESPO_CUDA_TRY(cudaGetLastError());
+  return ESPO_OK;
 }
 
 // ---------------------------------------------------------------------------------------
 // Per-device workspace, grown on demand.
 // ---------------------------------------------------------------------------------------
 struct AdvPool {
+  int sm_count = 0;
   void* arena = nullptr;
   int cap_B = 0;
   long long cap_chunks = 0;
-  unsigned epoch = 0;
   AdvWorkspace ws{};
 };
 constexpr int kMaxDevices = 64;
@@ -318,15 +374,14 @@ static int ensure_pool(int dev, int B, long long nchunks, AdvPool** out) {
     }
     size_t off = 0;
     auto carve = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    const size_t o_off = carve(8 * ((size_t)nb + 1)), o_cf = carve(4 * (size_t)nc), o_fl = carve(4 * (size_t)nc);
-    const size_t o_ag = carve(16 * (size_t)nc), o_fi = carve(8 * (size_t)nc), o_ct = carve(8), o_st = carve(4);
+    const size_t o_off = carve(8 * ((size_t)nb + 1)), o_cf = carve(4 * (size_t)nc), o_st = carve(4);
+    if (!p.sm_count) ESPO_CUDA_TRY(cudaDeviceGetAttribute(&p.sm_count, cudaDevAttrMultiProcessorCount, dev));
     ESPO_CUDA_TRY(cudaMalloc(&p.arena, off));
     ESPO_CUDA_TRY(cudaMemset(p.arena, 0, off));
     unsigned char* b = static_cast<unsigned char*>(p.arena);
-    p.ws.offsets = (long long*)(b + o_off); p.ws.chunk_first = (int*)(b + o_cf); p.ws.flag = (unsigned*)(b + o_fl);
-    p.ws.agg = (double2*)(b + o_ag); p.ws.fin = (double*)(b + o_fi); p.ws.counters = (unsigned*)(b + o_ct);
+    p.ws.offsets = (long long*)(b + o_off); p.ws.chunk_first = (int*)(b + o_cf);
     p.ws.status = (unsigned*)(b + o_st);
-    p.cap_B = nb; p.cap_chunks = nc; p.epoch = 0;
+    p.cap_B = nb; p.cap_chunks = nc;
   }
   *out = &p;
   return ESPO_OK;
@@ -341,11 +396,7 @@ constexpr int kNoAllocMaxB = ESPO_NOALLOC_MAX_B;
 constexpr long long kNoAllocMaxChunks = (ESPO_NOALLOC_MAX_TOKENS + kAdvChunk - 1) / kAdvChunk;
 constexpr size_t kNaOffOffsets = 0;
 constexpr size_t kNaOffChunkFirst = kNaOffOffsets + ((8 * ((size_t)kNoAllocMaxB + 1) + 255) / 256) * 256;
-constexpr size_t kNaOffFlag = kNaOffChunkFirst + 4 * (size_t)kNoAllocMaxChunks;
-constexpr size_t kNaOffAgg = kNaOffFlag + 4 * (size_t)kNoAllocMaxChunks;
-constexpr size_t kNaOffFin = kNaOffAgg + 16 * (size_t)kNoAllocMaxChunks;
-constexpr size_t kNaOffCounters = kNaOffFin + 8 * (size_t)kNoAllocMaxChunks;
-constexpr size_t kNaOffStatus = kNaOffCounters + 256;
+constexpr size_t kNaOffStatus = kNaOffChunkFirst + 4 * (size_t)kNoAllocMaxChunks;
 constexpr size_t kNoAllocBytes = kNaOffStatus + 256;
 static_assert(kNoAllocMaxChunks % 64 == 0, "keeps every sub-array 256-byte aligned");
 
@@ -353,7 +404,7 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
 struct NoAllocSlot {
   unsigned char* base = nullptr;   // device address of g_noalloc_scratch on this device
-  unsigned epoch = 0;
+  int sm_count = 0;
 };
 static NoAllocSlot g_noalloc[kMaxDevices];
 
@@ -383,36 +434,22 @@ int espo_advantages_noalloc(const float* rewards, const float* values, const int
     // In host code the array's name is only a handle; the kernels need its address on this device.
     void* p = nullptr;
     ESPO_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    ESPO_CUDA_TRY(cudaDeviceGetAttribute(&slot.sm_count, cudaDevAttrMultiProcessorCount, dev));
     slot.base = static_cast<unsigned char*>(p);
-    slot.epoch = 0;
   }
   cudaStream_t s = (cudaStream_t)stream;
   unsigned char* b = slot.base;
-  if (++slot.epoch >= (1u << 30)) {   // the descriptors' flags carry the epoch; start over before it wraps
-    ESPO_CUDA_TRY(cudaMemsetAsync(b + kNaOffFlag, 0, 4 * (size_t)kNoAllocMaxChunks, s));
-    slot.epoch = 1;
-  }
-  // The array keeps whatever the previous call left: the chunk tickets must start at zero even if
-  // that call was cut short, and the built-in status word is only ever OR-ed into.
-  ESPO_CUDA_TRY(cudaMemsetAsync(b + kNaOffCounters, 0, 8, s));
+  // The array keeps whatever the previous call left.  Nothing in it has to start at zero: the preparation
+  // kernel rewrites every offset and chunk owner this call reads, and the built-in status word is only OR-ed into.
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
   a.gamma = (double)gamma; a.gl = (double)gamma * (double)lambda;
   a.r_fail = r_fail;
-  a.epoch4 = slot.epoch << 2;
   a.ws.offsets = (long long*)(b + kNaOffOffsets);
   a.ws.chunk_first = (int*)(b + kNaOffChunkFirst);
-  a.ws.flag = (unsigned*)(b + kNaOffFlag);
-  a.ws.agg = (double2*)(b + kNaOffAgg);
-  a.ws.fin = (double*)(b + kNaOffFin);
-  a.ws.counters = (unsigned*)(b + kNaOffCounters);
   a.ws.status = status_out ? status_out : (unsigned*)(b + kNaOffStatus);
-  espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
-  ESPO_CUDA_TRY(cudaGetLastError());
-  espo_adv_scan_kernel<<<(unsigned)nchunks, kAdvThreads, 0, s>>>(a);
-  ESPO_CUDA_TRY(cudaGetLastError());
-  return ESPO_OK;
+  return launch_advantages(a, slot.sm_count, s);
 }
 
 int espo_advantages_reserve(int32_t max_B, int64_t max_tokens) {
@@ -444,22 +481,13 @@ int espo_advantages(const float* rewards, const float* values, const int32_t* le
   int rc = ensure_pool(dev, B, nchunks, &p);
   if (rc != ESPO_OK) return rc;
   cudaStream_t s = (cudaStream_t)stream;
-  if (++p->epoch >= (1u << 30)) {   // flags carry the epoch; start over before it wraps
-    ESPO_CUDA_TRY(cudaMemsetAsync(p->ws.flag, 0, 4 * (size_t)p->cap_chunks, s));
-    p->epoch = 1;
-  }
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
   a.gamma = (double)gamma; a.gl = (double)gamma * (double)lambda;
   a.r_fail = r_fail;
-  a.epoch4 = p->epoch << 2;
   a.ws = p->ws;
-  espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
-  ESPO_CUDA_TRY(cudaGetLastError());
-  espo_adv_scan_kernel<<<(unsigned)nchunks, kAdvThreads, 0, s>>>(a);
-  ESPO_CUDA_TRY(cudaGetLastError());
-  return ESPO_OK;
+  return launch_advantages(a, p->sm_count, s);
 }
 
 int espo_advantages_status(uint32_t* host_out, void* stream) {
