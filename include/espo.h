@@ -203,7 +203,7 @@ int espo_advantages_status(uint32_t* host_out, void* stream);
  * own pools at start-up, so that a cudaMalloc issued by a library fails; and a training loop
  * that cannot afford the device-wide synchronisation that cudaMalloc/cudaFree imply.  This call
  * never calls cudaMalloc, cudaFree or any other allocating routine: its scratch is a fixed
- * array of about 0.3 MB that is part of the library image, so every device that loads the
+ * array of about 50 KB that is part of the library image, so every device that loads the
  * library holds that array until the process exits.
  *
  * Arguments are those of espo_advantages, plus
@@ -214,9 +214,10 @@ int espo_advantages_status(uint32_t* host_out, void* stream);
  * ESPO_ERR_CAPACITY and nothing is launched.
  * The first call on each device looks up the scratch array's device address (with that device
  * current) and remembers it; make that first call outside any stream capture.
- * All calls on a device share the one array and it keeps the previous call's contents; the
- * call itself clears the part that has to start at zero.  Two calls that overlap on the
- * device (different streams, no dependency) race on it: serialise them.
+ * All calls on a device share the one array and it keeps the previous call's contents; no
+ * part of it has to start at zero, because each call rewrites every entry it later reads.
+ * Two calls that overlap on the device (different streams, no dependency) race on it:
+ * serialise them.
  * Errors: BAD_SHAPE, CAPACITY, NULL, ALIGN (16-byte arrays), BAD_PARAM, CUDA. */
 int espo_advantages_noalloc(const float* rewards, const float* values, const int32_t* lengths,
                             const uint8_t* stopped, int32_t B, int64_t total_tokens,
