@@ -202,6 +202,14 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// ln of a sum of exponentials that is known to lie in [1, 1024 * 32]: lg2.approx has an absolute error below
+// 2^-22 on the mantissa's logarithm, i.e. below 2e-7 here -- two orders under the sampler's tie margin.
+__device__ __forceinline__ float log_sum(float s) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(s));
+  return y * 0.6931471805599453f;
+}
+
 __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
   uint32_t c;
   asm("max.bf16x2 %0, %1, %2;" : "=r"(c) : "r"(a), "r"(b));

@@ -317,7 +317,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       if (id >= 0 && (best_i < 0 || sc > best)) { best = sc; best_i = id; }
     } else {
       const float ln_e = noise ? noise[b] : logf(expo_at(ds, 2u, (uint32_t)b));
-      const float sc = fmaf(m_b, a.inv_temp, logf(s_b) - ln_e);
+      const float sc = fmaf(m_b, a.inv_temp, log_sum(s_b) - ln_e);
       if (best_i < 0 || sc > best) { best = sc; best_i = b; }
     }
   };
@@ -389,6 +389,8 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       for (int i = 0; i < kSubIds; ++i) x[i] = (i < n_here) ? load_logit<ES>(row_base, sub_lo + i) : NINF;
     }
 
+    // the sub-block's noise does not depend on the data: drawn while the loads above are in flight
+    const float ln_e1 = a.greedy ? 0.f : logf(expo_at(ds, 1u, (uint32_t)(sub_lo >> 5)));   // index = global sub-block number
     if (a.greedy) {
       // first id equal to the maximum
       int first = -1;
@@ -406,9 +408,8 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       int j = -1;
       if (m_j > NINF) {
         const float s_j = sum_exp2_32(x, m_j, a.k2);
-        const uint32_t jg = (uint32_t)(sub_lo >> 5);   // global sub-block number
-        sc = fmaf(m_j, a.inv_temp, logf(s_j / expo_at(ds, 1u, jg)));
-        j = (int)jg;
+        sc = fmaf(m_j, a.inv_temp, log_sum(s_j) - ln_e1);
+        j = sub_lo >> 5;
       }
       warp_argmax(sc, j);
       const int sub_pick = max(j, blk_lo >> 5);        // j < 0 cannot happen: the block has a finite id
