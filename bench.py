@@ -180,6 +180,7 @@ def main():
     ap.add_argument("--sampler", default="hier", choices=["hier", "flat"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the single-step timings at other shapes")
+    ap.add_argument("--eager", action="store_true", help="launch every step separately instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = args.steps or 4
@@ -229,6 +230,28 @@ def main():
         for i in range(n_steps):
             espo.espo_step(bufs[i % N_BUFFERS], values, state, params, tokens, stop)
 
+    # The decode loop is launch-latency sensitive (one 35 us kernel per step), so the timed rollout replays a CUDA
+    # graph of GRAPH_STEPS consecutive steps (the remainder, and everything with --eager, is launched one by one).
+    graph, graph_steps = None, 0
+    if not args.eager and K >= 2 * N_BUFFERS:
+        graph_steps = min(400, K) // N_BUFFERS * N_BUFFERS
+        graph = torch.cuda.CUDAGraph()
+        cap_stream = torch.cuda.Stream()
+        cap_stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cap_stream):
+            rollout(N_BUFFERS)                      # warm the capture stream
+            with torch.cuda.graph(graph, stream=cap_stream):
+                rollout(graph_steps)
+        torch.cuda.current_stream().wait_stream(cap_stream)
+
+    def timed_rollout(n_steps):
+        done = 0
+        if graph is not None:
+            while done + graph_steps <= n_steps:
+                graph.replay()
+                done += graph_steps
+        rollout(n_steps - done)
+
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
@@ -246,7 +269,7 @@ def main():
     ev0, ev1, ev2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
     t_wall0 = time.time()
     ev0.record()
-    rollout(K)
+    timed_rollout(K)
     ev1.record()
     espo.espo_advantages(adv_r, adv_v, adv_len, adv_stopped, 1.0, 0.95, -1.0, adv_out)
     ev2.record()
@@ -279,6 +302,7 @@ def main():
             "workload": f"rollout-batch scale: B={B} trajectories per GPU, V={V}, bf16 logits ~N(0,3) + 5 Zipf peaks, "
                         f"temperature 1.0, {args.sampler} Philox Gumbel-max sampler, full active set; timed region = "
                         f"{K} decode steps + 1 advantage pass over the {adv_tokens} tokens generated",
+            "launch": ("eager launches" if graph is None else f"CUDA graph of {graph_steps} steps replayed"),
             "l2": f"{N_BUFFERS} logit buffers of {bytes_per_launch / 1e6:.1f} MB rotate (each larger than the 126 MB L2)",
             "parallelism": f"rows sharded over {world} GPU(s), no collective",
             "stopped_rows": n_stopped, "device_status": dev_status,

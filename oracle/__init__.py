@@ -98,6 +98,9 @@ def lib():
             fn = getattr(L, name)
             fn.argtypes = [dp, dp, ip, u8p, C.c_int32, C.c_double, C.c_double, C.c_double, dp]
             fn.restype = None
+        L.espo_oracle_end_batch.argtypes = [C.POINTER(RowState), C.c_int32, C.c_double, C.c_double, C.c_double,
+                                            C.c_double, C.c_double, C.c_int32, dp, dp, dp, dp]
+        L.espo_oracle_end_batch.restype = None
         L.espo_oracle_advantages_f32.argtypes = [fp, fp, ip, u8p, C.c_int32, C.c_double, C.c_double,
                                                  C.c_double, dp, C.c_int32]
         L.espo_oracle_advantages_f32.restype = None
@@ -169,6 +172,16 @@ class Rollout:
             None if rid is None else _ptr(rid, C.c_int32), n_rows, self.seed, self.batch_id,
             C.byref(params), self.states, outs, int(n_threads))
         return outs
+
+    def end_batch(self, mu_g, sigma2_g, beta, alpha_ema=0.99, eta_beta=0.1, tau=0.25, beta_min=0.0, beta_max=1e30,
+                  first_update=False):
+        """Batch-boundary update (Eq. 7-8, 12).  Returns (mu_g, sigma2_g, beta, stats[6])."""
+        m, v, b = C.c_double(mu_g), C.c_double(sigma2_g), C.c_double(beta)
+        out = (C.c_double * 6)()
+        lib().espo_oracle_end_batch(self.states, self.capacity, float(alpha_ema), float(eta_beta), float(tau),
+                                    float(beta_min), float(beta_max), int(bool(first_update)),
+                                    C.byref(m), C.byref(v), C.byref(b), out)
+        return m.value, v.value, b.value, list(out)
 
     def snapshot(self, slot: int) -> RowState:
         s = RowState()

@@ -12,6 +12,8 @@
 //   * smoothed cumulative regret z_t = a_s z_{t-1} + (1-a_s) g~_t, z_0 = 0        (Sec. 4.2, Eq. 10)
 //   * value-gated stop  z_t > beta * max(V_phi(s_t), eps), only after warm-up     (Sec. 4.3, Eq. 11; Algorithm 1)
 //   * failure transition r_{T_stop} = r_fail, nothing bootstrapped past the end   (Sec. 4.4, Eq. 13)
+//   * batch statistics  mu_g, sigma_g^2: EMA of the batch mean / variance of g    (Sec. 4.2, Eq. 7-8)
+//   * threshold control beta <- clip(beta + eta (rho_stop - tau), b_min, b_max)   (Sec. 4.3, Eq. 12)
 //   * TD error and GAE  delta_t = r_t + gamma V(s_{t+1}) - V(s_t),
 //                       A_t = sum_l (gamma lambda)^l delta_{t+l}                  (Sec. 3, Eq. 4-5)
 //
@@ -455,6 +457,50 @@ void espo_oracle_advantages_f32(const float* rewards, const float* values,
   for (int32_t k = 0; k < n_threads; ++k)
     pool.emplace_back(work, (int32_t)((int64_t)B * k / n_threads), (int32_t)((int64_t)B * (k + 1) / n_threads));
   for (auto& th : pool) th.join();
+}
+
+// ---------------------------------------------------------------------------
+// Batch boundary (Sec. 4.2, Eq. 7-8; Sec. 4.3, Eq. 12).  After a rollout batch:
+//   g_B      = every regret value generated in the batch (all tokens of all
+//              trajectories that took part, stop-step tokens included)
+//   mu_g     <- a_ema mu_g     + (1 - a_ema) mean(g_B)
+//   sigma_g2 <- a_ema sigma_g2 + (1 - a_ema) Var(g_B)        (population variance)
+//   beta     <- clip(beta + eta_beta (rho_stop - tau), beta_min, beta_max)
+// rho_stop = stopped trajectories / trajectories that took part (t > 0).  With
+// first_update != 0 the statistics are set to the batch values (nothing to average with
+// yet).  An empty batch changes nothing.  out6 = {mean, var, rho_stop, tokens, trajectories,
+// stopped}.
+// ---------------------------------------------------------------------------
+void espo_oracle_end_batch(const espo_oracle_row_state* states, int32_t n_slots,
+                           double alpha_ema, double eta_beta, double tau, double beta_min, double beta_max,
+                           int32_t first_update, double* mu_g, double* sigma2_g, double* beta, double* out6) {
+  double sg = 0.0, sg2 = 0.0;
+  int64_t n_tok = 0, n_traj = 0, n_stop = 0;
+  for (int32_t i = 0; i < n_slots; ++i) {
+    if (states[i].t <= 0) continue;
+    sg += states[i].sum_g;
+    sg2 += states[i].sum_g2;
+    n_tok += states[i].n_tokens;
+    n_traj += 1;
+    if (states[i].status == ORACLE_STOPPED) n_stop += 1;
+  }
+  double mean = 0.0, var = 0.0, rho = 0.0;
+  if (n_tok > 0) {
+    mean = sg / (double)n_tok;
+    var = sg2 / (double)n_tok - mean * mean;
+    if (var < 0.0) var = 0.0;
+    rho = (double)n_stop / (double)n_traj;
+    if (first_update) { *mu_g = mean; *sigma2_g = var; }
+    else {
+      *mu_g = alpha_ema * (*mu_g) + (1.0 - alpha_ema) * mean;
+      *sigma2_g = alpha_ema * (*sigma2_g) + (1.0 - alpha_ema) * var;
+    }
+    double b = *beta + eta_beta * (rho - tau);
+    if (b < beta_min) b = beta_min;
+    if (b > beta_max) b = beta_max;
+    *beta = b;
+  }
+  if (out6) { out6[0] = mean; out6[1] = var; out6[2] = rho; out6[3] = (double)n_tok; out6[4] = (double)n_traj; out6[5] = (double)n_stop; }
 }
 
 }  // extern "C"

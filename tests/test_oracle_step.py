@@ -344,3 +344,40 @@ def test_float32_entry_point_agrees():
     for r in range(5):
         assert (a[r].token, a[r].stop) == (b[r].token, b[r].stop)
         assert a[r].z == b[r].z and a[r].logp == b[r].logp
+
+
+# --------------------------------------------------------------------------- batch boundary (Eq. 7-8, 12)
+
+
+def test_end_batch_matches_numpy_statistics_and_the_controller_formula():
+    # every regret value of a small rollout is collected by hand; the EMA targets are numpy's mean / population variance
+    rng = _rng(40)
+    B, V, T = 6, 400, 9
+    ro = oracle.Rollout(B, seed=3)
+    p = oracle.make_params(temperature=1.0, mu_g=0.5, sigma2_g=1.0, alpha_s=0.5, beta=0.8, eps=0.2, t_max=T)
+    gs, stopped = [], set()
+    for t in range(T):
+        x = _peaked_logits(rng, B, V)
+        outs = ro.step(x, rng.uniform(0.0, 1.0, size=B), p)
+        for r in range(B):
+            if outs[r].token >= 0:
+                gs.append(outs[r].g)
+            if outs[r].stop:
+                stopped.add(r)
+    assert 0 < len(stopped) < B
+    gs = np.array(gs)
+    mu, s2, beta, st = ro.end_batch(2.0, 3.0, 7.0, alpha_ema=0.9, eta_beta=0.1, tau=0.25, beta_min=0.0, beta_max=10.0)
+    assert st[3] == len(gs) and st[4] == B and st[5] == len(stopped)
+    assert abs(st[0] - gs.mean()) < 1e-12 and abs(st[1] - gs.var()) < 1e-12
+    assert abs(mu - (0.9 * 2.0 + 0.1 * gs.mean())) < 1e-12
+    assert abs(s2 - (0.9 * 3.0 + 0.1 * gs.var())) < 1e-12
+    assert abs(beta - (7.0 + 0.1 * (len(stopped) / B - 0.25))) < 1e-12
+    # first update: the statistics are the batch's own; the clip bounds hold
+    mu, s2, beta, _ = ro.end_batch(2.0, 3.0, 7.0, eta_beta=100.0, tau=0.0, beta_max=7.5, first_update=True)
+    assert abs(mu - gs.mean()) < 1e-12 and abs(s2 - gs.var()) < 1e-12 and beta == 7.5
+    _, _, beta, _ = ro.end_batch(2.0, 3.0, 7.0, eta_beta=100.0, tau=1.0, beta_min=0.0)
+    assert beta == 0.0
+    # stop rate on target leaves beta alone; an empty batch changes nothing
+    _, _, beta, _ = ro.end_batch(2.0, 3.0, 7.0, tau=len(stopped) / B)
+    assert beta == 7.0
+    assert oracle.Rollout(4, seed=1).end_batch(2.0, 3.0, 7.0)[:3] == (2.0, 3.0, 7.0)
