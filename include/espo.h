@@ -160,6 +160,23 @@ int espo_set_launch_config(espo_state* st, int32_t consumer_warps, int32_t stage
  * n_active_out (device int32 [1]).  Enqueued on `stream`. */
 int espo_compact_active(espo_state* st, int32_t* row_ids_out, int32_t* n_active_out, void* stream);
 
+/* Batch boundary (Sec. 4.2, Eq. 7-8 and Sec. 4.3, Eq. 12), to be called after the last step of a
+ * rollout batch and before espo_reset_state.  Over the slots that took part (t > 0) it forms, on
+ * the device, the mean and the population variance of every regret value g generated in the
+ * batch (stop-step tokens included) and the empirical stop rate rho = stopped / took part, then
+ *   mu_g     <- alpha_ema mu_g     + (1 - alpha_ema) mean      (set to mean if first_update)
+ *   sigma2_g <- alpha_ema sigma2_g + (1 - alpha_ema) variance  (set to variance if first_update)
+ *   beta     <- clip(beta + eta_beta (rho - tau), beta_min, beta_max)
+ * reading the old values from *params_inout (host) and writing the new ones back to it; the
+ * other fields are left alone.  The paper's values: alpha_ema 0.99, eta_beta 0.1, tau 0.25,
+ * beta_min 0; it names beta_max without a value.  A batch without tokens changes nothing.
+ *   stats_out  host double [6] or NULL: mean, variance, rho, tokens, trajectories, stopped
+ * Synchronises `stream`.  Errors: NULL, BAD_PARAM (alpha_ema outside [0,1], NaN, beta_min >
+ * beta_max), CUDA. */
+int espo_end_batch(espo_state* st, float alpha_ema, float eta_beta, float tau, float beta_min,
+                   float beta_max, int32_t first_update, espo_params* params_inout,
+                   double* stats_out, void* stream);
+
 /* Copy the sticky device status word (ESPO_DEV_* bits) to *host_out.  Synchronises `stream`. */
 int espo_state_status(espo_state* st, uint32_t* host_out, void* stream);
 

@@ -70,6 +70,7 @@ def lib():
         L.espo_state_view.argtypes = [vp] + [C.POINTER(vp)] * 9
         L.espo_compact_active.argtypes = [vp, vp, vp, vp]
         L.espo_state_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        L.espo_end_batch.argtypes = [vp, f32, f32, f32, f32, f32, i32, C.POINTER(espo_params), C.POINTER(C.c_double), vp]
         L.espo_advantages.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp]
         L.espo_advantages_noalloc.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp]
         L.espo_advantages_reserve.argtypes = [i32, i64]
@@ -78,7 +79,7 @@ def lib():
         L.espo_strerror.restype = C.c_char_p
         L.espo_last_cuda_error.argtypes = []
         for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_state_view",
-                  "espo_compact_active", "espo_state_status", "espo_advantages", "espo_advantages_reserve",
+                  "espo_compact_active", "espo_state_status", "espo_end_batch", "espo_advantages", "espo_advantages_reserve",
                   "espo_advantages_status", "espo_advantages_noalloc", "espo_last_cuda_error"):
             getattr(L, n).restype = C.c_int
         _lib = L
@@ -202,6 +203,18 @@ def espo_compact_active(state: EspoState, row_ids_out: torch.Tensor, n_active_ou
         raise ValueError("row_ids_out must hold capacity entries and n_active_out one")
     _check(lib().espo_compact_active(state.handle, _dev_ptr(row_ids_out, "row_ids_out"),
                                      _dev_ptr(n_active_out, "n_active_out"), _stream(stream)), "espo_compact_active")
+
+
+def espo_end_batch(state: EspoState, params: espo_params, alpha_ema: float = 0.99, eta_beta: float = 0.1,
+                   tau: float = 0.25, beta_min: float = 0.0, beta_max: float = 3.0e38, first_update: bool = False,
+                   stream=None) -> dict:
+    """Batch-boundary update (Eq. 7-8, 12): rewrites params.mu_g, params.sigma2_g and params.beta in place and
+    returns the batch statistics; see ``espo.h``.  Synchronises the stream."""
+    out = (C.c_double * 6)()
+    _check(lib().espo_end_batch(state.handle, alpha_ema, eta_beta, tau, beta_min, beta_max, int(bool(first_update)),
+                                C.byref(params), out, _stream(stream)), "espo_end_batch")
+    return {"mean_g": out[0], "var_g": out[1], "stop_rate": out[2], "tokens": int(out[3]), "trajectories": int(out[4]),
+            "stopped": int(round(out[5]))}
 
 
 def espo_state_status(state: EspoState, stream=None) -> int:

@@ -798,6 +798,7 @@ struct espo_state {
   double *sum_g, *sum_g2;
   float4* records;
   unsigned *ticket, *dev_status;
+  double* batch_out;   // [8] result of espo_end_batch
 };
 
 namespace espo {
@@ -828,6 +829,64 @@ __global__ void espo_compact_kernel(const uint8_t* __restrict__ status, int capa
     __syncthreads();
   }
   if (threadIdx.x == 0) *n_out = base;
+}
+
+// Batch boundary (Eq. 7-8, 12): reduces the per-slot sums over the slots that took part (t > 0) and applies the
+// EMA and the proportional controller.  One CTA; out = {mu_g, sigma2_g, beta, mean, var, rho_stop, tokens,
+// trajectories} -- stopped trajectories = rho_stop * trajectories.
+struct EndBatchArgs {
+  const double *sum_g, *sum_g2;
+  const int32_t* t;
+  const uint8_t* status;
+  int capacity;
+  double mu_g, sigma2_g, beta, alpha_ema, eta_beta, tau, beta_min, beta_max;
+  int first_update;
+  double* out;
+};
+
+__global__ void __launch_bounds__(1024) espo_end_batch_kernel(const EndBatchArgs e) {
+  __shared__ double red[5][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double acc[5] = {0.0, 0.0, 0.0, 0.0, 0.0};   // sum g, sum g^2, tokens, trajectories, stopped
+  for (int i = threadIdx.x; i < e.capacity; i += blockDim.x) {
+    const int ti = e.t[i];
+    if (ti > 0) {
+      acc[0] += e.sum_g[i]; acc[1] += e.sum_g2[i]; acc[2] += (double)ti; acc[3] += 1.0;
+      if (e.status[i] == ESPO_ROW_STOPPED) acc[4] += 1.0;
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 5; ++k) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc[k] += __shfl_xor_sync(kFullMask, acc[k], o);
+    if (lane == 0) red[k][warp] = acc[k];
+  }
+  __syncthreads();
+  if (warp == 0) {
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+      double v = (lane < (int)(blockDim.x >> 5)) ? red[k][lane] : 0.0;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+      acc[k] = v;
+    }
+    if (lane == 0) {
+      double mu = e.mu_g, s2 = e.sigma2_g, beta = e.beta, mean = 0.0, var = 0.0, rho = 0.0;
+      if (acc[2] > 0.0) {
+        mean = acc[0] / acc[2];
+        var = fmax(acc[1] / acc[2] - mean * mean, 0.0);
+        rho = acc[4] / acc[3];
+        if (e.first_update) { mu = mean; s2 = var; }
+        else {
+          mu = e.alpha_ema * mu + (1.0 - e.alpha_ema) * mean;
+          s2 = e.alpha_ema * s2 + (1.0 - e.alpha_ema) * var;
+        }
+        beta = fmin(fmax(beta + e.eta_beta * (rho - e.tau), e.beta_min), e.beta_max);
+      }
+      e.out[0] = mu; e.out[1] = s2; e.out[2] = beta; e.out[3] = mean; e.out[4] = var; e.out[5] = rho;
+      e.out[6] = acc[2]; e.out[7] = acc[3];
+    }
+  }
 }
 
 using StepKernel = void (*)(const StepArgs);
@@ -877,7 +936,7 @@ int espo_init_state(espo_state** out, int32_t capacity, int32_t V, uint64_t seed
   const size_t o_t = carve(4 * cap), o_ts = carve(4 * cap), o_st = carve(cap);
   const size_t o_sg = carve(8 * cap), o_sg2 = carve(8 * cap);
   const size_t o_rec = carve(sizeof(float4) * cap * (size_t)st->nblk);
-  const size_t o_tk = carve(4 * cap), o_ds = carve(4);
+  const size_t o_tk = carve(4 * cap), o_ds = carve(4), o_bo = carve(8 * 8);
   st->arena_bytes = off;
   e = cudaMalloc(&st->arena, st->arena_bytes);
   if (e != cudaSuccess) { delete st; return record_cuda_error(e); }
@@ -886,6 +945,7 @@ int espo_init_state(espo_state** out, int32_t capacity, int32_t V, uint64_t seed
   st->logp = (float*)(base + o_lp); st->t = (int32_t*)(base + o_t); st->t_stop = (int32_t*)(base + o_ts);
   st->status = (uint8_t*)(base + o_st); st->sum_g = (double*)(base + o_sg); st->sum_g2 = (double*)(base + o_sg2);
   st->records = (float4*)(base + o_rec); st->ticket = (unsigned*)(base + o_tk); st->dev_status = (unsigned*)(base + o_ds);
+  st->batch_out = (double*)(base + o_bo);
 
   for (int es = 2; es <= 4; es += 2)
     for (int sm = 0; sm < 2; ++sm)
@@ -1048,6 +1108,34 @@ int espo_compact_active(espo_state* st, int32_t* row_ids_out, int32_t* n_active_
   if (!st || !row_ids_out || !n_active_out) return ESPO_ERR_NULL;
   espo::espo_compact_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>(st->status, st->capacity, row_ids_out, n_active_out);
   ESPO_CUDA_TRY(cudaGetLastError());
+  return ESPO_OK;
+}
+
+int espo_end_batch(espo_state* st, float alpha_ema, float eta_beta, float tau, float beta_min, float beta_max,
+                   int32_t first_update, espo_params* params_inout, double* stats_out, void* stream) {
+  if (!st || !params_inout) return ESPO_ERR_NULL;
+  if (!(alpha_ema >= 0.f && alpha_ema <= 1.f) || isnan(eta_beta) || isnan(tau) || isnan(beta_min) || isnan(beta_max) ||
+      beta_min > beta_max || isnan(params_inout->mu_g) || isnan(params_inout->sigma2_g) || isnan(params_inout->beta))
+    return ESPO_ERR_BAD_PARAM;
+  espo::EndBatchArgs e;
+  e.sum_g = st->sum_g; e.sum_g2 = st->sum_g2; e.t = st->t; e.status = st->status; e.capacity = st->capacity;
+  e.mu_g = params_inout->mu_g; e.sigma2_g = params_inout->sigma2_g; e.beta = params_inout->beta;
+  e.alpha_ema = alpha_ema; e.eta_beta = eta_beta; e.tau = tau; e.beta_min = beta_min; e.beta_max = beta_max;
+  e.first_update = first_update != 0;
+  e.out = st->batch_out;
+  cudaStream_t s = (cudaStream_t)stream;
+  espo::espo_end_batch_kernel<<<1, 1024, 0, s>>>(e);
+  ESPO_CUDA_TRY(cudaGetLastError());
+  double host[8];
+  ESPO_CUDA_TRY(cudaMemcpyAsync(host, st->batch_out, sizeof(host), cudaMemcpyDeviceToHost, s));
+  ESPO_CUDA_TRY(cudaStreamSynchronize(s));
+  params_inout->mu_g = (float)host[0];
+  params_inout->sigma2_g = (float)host[1];
+  params_inout->beta = (float)host[2];
+  if (stats_out) {
+    stats_out[0] = host[3]; stats_out[1] = host[4]; stats_out[2] = host[5];
+    stats_out[3] = host[6]; stats_out[4] = host[7]; stats_out[5] = host[5] * host[7];
+  }
   return ESPO_OK;
 }
 

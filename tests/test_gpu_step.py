@@ -238,6 +238,31 @@ def test_compaction_and_shrinking_active_set():
     run.close()
 
 
+def test_end_batch_updates_statistics_and_beta_like_the_oracle():
+    # a short rollout in which some rows stop, then the batch-boundary update (Eq. 7-8, 12) on both sides
+    B, V, T = 40, 6000, 10
+    p = espo.make_params(temperature=1.0, mu_g=0.5, sigma2_g=1.0, alpha_s=0.6, beta=1.0, eps=0.2)
+    run = ParityRun(B + 3, V, p, seed=21)            # three slots never take part
+    for t in range(T):
+        x = synth.logits_batch(B, V, dtype=torch.bfloat16, sd=2.5, seed=700 + t)
+        vals = torch.rand(B, device="cuda", generator=torch.Generator("cuda").manual_seed(50 + t))
+        run.step(x, vals)
+    assert run.stats.stops > 0 and not run.dropped
+    for first in (False, True):
+        q = espo.make_params(mu_g=2.0, sigma2_g=3.0, beta=7.0)
+        st = espo.espo_end_batch(run.state, q, alpha_ema=0.9, eta_beta=0.5, tau=0.25, beta_min=0.0, beta_max=7.2,
+                                 first_update=first)
+        mu, s2, beta, ost = run.ro.end_batch(2.0, 3.0, 7.0, alpha_ema=0.9, eta_beta=0.5, tau=0.25, beta_min=0.0,
+                                             beta_max=7.2, first_update=first)
+        assert close(q.mu_g, mu) and close(q.sigma2_g, s2) and close(q.beta, beta)
+        assert close(st["mean_g"], ost[0]) and close(st["var_g"], ost[1]) and close(st["stop_rate"], ost[2])
+        assert (st["tokens"], st["trajectories"], st["stopped"]) == (int(ost[3]), B, int(ost[5]))
+    with pytest.raises(espo.EspoError) as e:
+        espo.espo_end_batch(run.state, p, alpha_ema=1.5)
+    assert e.value.code == espo.ESPO_ERR_BAD_PARAM
+    run.close()
+
+
 def test_reset_state_starts_a_new_batch():
     B, V = 4, 4096
     p = espo.make_params(mu_g=1.0, sigma2_g=2.0, beta=100.0)
