@@ -25,6 +25,7 @@ _lib = None
 
 ACTIVE, STOPPED, EOS, TMAX, BAD = 0, 1, 2, 3, 4
 SAMPLER_FLAT, SAMPLER_HIER = 0, 1
+STOP_ESPO, STOP_VALUE_ONLY, STOP_REGRET_ONLY, STOP_RANDOM = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -45,7 +46,8 @@ class Params(C.Structure):
     _fields_ = [("temperature", C.c_double), ("mu_g", C.c_double), ("sigma2_g", C.c_double),
                 ("delta", C.c_double), ("clip_c", C.c_double), ("alpha_s", C.c_double),
                 ("beta", C.c_double), ("eps", C.c_double), ("warmup_complete", C.c_int32),
-                ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32)]
+                ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32),
+                ("stop_mode", C.c_int32), ("shadow", C.c_int32), ("tau", C.c_double), ("p_random", C.c_double)]
 
 
 class RowState(C.Structure):
@@ -62,10 +64,11 @@ class StepOut(C.Structure):
 
 
 def make_params(temperature=1.0, mu_g=0.0, sigma2_g=1.0, delta=1e-8, clip_c=10.0, alpha_s=0.9,
-                beta=7.0, eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=SAMPLER_FLAT) -> Params:
+                beta=7.0, eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=SAMPLER_FLAT,
+                stop_mode=0, shadow=0, tau=0.0, p_random=0.0) -> Params:
     return Params(float(temperature), float(mu_g), float(sigma2_g), float(delta), float(clip_c),
                   float(alpha_s), float(beta), float(eps), int(warmup_complete), int(t_max),
-                  int(eos_token), int(sampler))
+                  int(eos_token), int(sampler), int(stop_mode), int(shadow), float(tau), float(p_random))
 
 
 def lib():

@@ -153,6 +153,13 @@ struct espo_oracle_params {
   int32_t t_max;                           // horizon T_max
   int32_t eos_token;                       // -1: none
   int32_t sampler;                         // 0 flat, 1 hierarchical
+  // Stop rules of the ablation study (Sec. 6): 0 the method's rule (Eq. 11); 1 value only, V_phi(s_t) < tau;
+  // 2 regret only, z_t > tau; 3 random, with probability p_random per step.  shadow != 0: the first step at
+  // which the rule holds is recorded in t_stop but the trajectory is not ended (the analysis' "Original" curves).
+  int32_t stop_mode;
+  int32_t shadow;
+  double tau;
+  double p_random;
 };
 
 enum { ORACLE_ACTIVE = 0, ORACLE_STOPPED = 1, ORACLE_EOS = 2, ORACLE_TMAX = 3, ORACLE_BAD = 4 };
@@ -292,9 +299,14 @@ void espo_oracle_step_row(const double* logits, int64_t V, double value,
   // Eq. 10: updated on every step, warm-up or not (Algorithm 1 updates z before the gated test).
   const double z = p->alpha_s * st->z + (1.0 - p->alpha_s) * gt;
 
-  // Eq. 11, strict inequality; a NaN value estimate never stops.
+  // Eq. 11, strict inequality; a NaN value estimate never stops.  The ablation's rules replace the inequality.
   const double thr = p->beta * std::fmax(value, p->eps);
-  const bool fires = (p->warmup_complete != 0) && !std::isnan(value) && (z > thr);
+  bool rule = false;
+  if (p->stop_mode == 0) rule = !std::isnan(value) && (z > thr);
+  else if (p->stop_mode == 1) rule = !std::isnan(value) && (value < p->tau);
+  else if (p->stop_mode == 2) rule = (z > p->tau);
+  else rule = (uniform_for(dk, 3, 0) < p->p_random);       // one more draw of the step's Philox stream: level 3, index 0
+  const bool fires = (p->warmup_complete != 0) && rule;
 
   st->z = z;
   st->sum_g += g;
@@ -306,6 +318,9 @@ void espo_oracle_step_row(const double* logits, int64_t V, double value,
   int32_t stop = 0;
   if (p->eos_token >= 0 && token == p->eos_token) {
     st->status = ORACLE_EOS;
+  } else if (fires && p->shadow) {
+    if (st->t_stop < 0) st->t_stop = t_now;                // remembered, not acted upon
+    if (st->t >= p->t_max) st->status = ORACLE_TMAX;
   } else if (fires) {
     st->status = ORACLE_STOPPED;
     st->t_stop = t_now;

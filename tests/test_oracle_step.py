@@ -381,3 +381,69 @@ def test_end_batch_matches_numpy_statistics_and_the_controller_formula():
     _, _, beta, _ = ro.end_batch(2.0, 3.0, 7.0, tau=len(stopped) / B)
     assert beta == 7.0
     assert oracle.Rollout(4, seed=1).end_batch(2.0, 3.0, 7.0)[:3] == (2.0, 3.0, 7.0)
+
+
+# --------------------------------------------------------------------------- the ablation's stop rules (Sec. 6)
+
+
+def _rollout_with(mode_kwargs, T=12, B=5, V=300, seed=50, values=None):
+    rng = _rng(seed)
+    ro = oracle.Rollout(B, seed=9)
+    kw = dict(temperature=1.0, mu_g=0.5, sigma2_g=1.0, alpha_s=0.5, beta=0.8, eps=0.2, t_max=10**6)
+    kw.update(mode_kwargs)
+    p = oracle.make_params(**kw)
+    hist = []
+    for t in range(T):
+        x = _peaked_logits(rng, B, V)
+        v = rng.uniform(0.0, 1.0, size=B) if values is None else values[t]
+        outs = ro.step(x, v, p)
+        hist.append([(o.token, o.stop, o.z, float(v[r])) for r, o in enumerate(outs)])
+    return ro, hist
+
+
+def test_value_only_and_regret_only_rules_fire_exactly_on_their_inequality():
+    for mode, tau in ((oracle.STOP_VALUE_ONLY, 0.3), (oracle.STOP_REGRET_ONLY, 0.4)):
+        ro, hist = _rollout_with(dict(stop_mode=mode, tau=tau))
+        fired = 0
+        for step in hist:
+            for tok, stop, z, v in step:
+                if tok < 0:
+                    continue                      # already ended
+                want = (v < tau) if mode == oracle.STOP_VALUE_ONLY else (z > tau)
+                assert bool(stop) == want
+                fired += int(stop)
+        assert fired > 0
+    # the warm-up gate applies to every rule
+    _, hist = _rollout_with(dict(stop_mode=oracle.STOP_VALUE_ONLY, tau=2.0, warmup_complete=0))
+    assert not any(stop for step in hist for _, stop, _, _ in step)
+
+
+def test_random_rule_has_the_requested_rate_and_does_not_disturb_the_sampler():
+    _, base = _rollout_with(dict(stop_mode=oracle.STOP_ESPO, beta=1e9), T=6)
+    _, never = _rollout_with(dict(stop_mode=oracle.STOP_RANDOM, p_random=0.0), T=6)
+    _, always = _rollout_with(dict(stop_mode=oracle.STOP_RANDOM, p_random=1.0), T=6)
+    assert [[t for t, _, _, _ in s] for s in base] == [[t for t, _, _, _ in s] for s in never]   # same tokens
+    assert all(stop for _, stop, _, _ in always[0]) and all(t == -1 for t, _, _, _ in always[1])
+    # rate: 4000 independent (slot, step 0) draws at p = 0.25
+    B = 4000
+    ro = oracle.Rollout(B, seed=123)
+    p = oracle.make_params(stop_mode=oracle.STOP_RANDOM, p_random=0.25)
+    outs = ro.step(np.zeros((B, 8)), np.zeros(B), p)
+    k = sum(o.stop for o in outs)
+    assert abs(k - 1000) < 5 * math.sqrt(B * 0.25 * 0.75)
+
+
+def test_shadow_mode_records_the_first_firing_step_and_keeps_decoding():
+    T = 12
+    ro_a, hist_a = _rollout_with(dict(stop_mode=oracle.STOP_ESPO), T=T)
+    ro_s, hist_s = _rollout_with(dict(stop_mode=oracle.STOP_ESPO, shadow=1), T=T)
+    n_stopped = 0
+    for r in range(ro_a.capacity):
+        a, s = ro_a.states[r], ro_s.states[r]
+        assert s.status == oracle.ACTIVE and s.t == T            # never ended
+        assert s.t_stop == a.t_stop                               # same first firing step (or none)
+        n_stopped += int(a.t_stop >= 0)
+        upto = T if a.t_stop < 0 else a.t_stop + 1
+        assert [h[r][0] for h in hist_s[:upto]] == [h[r][0] for h in hist_a[:upto]]   # same tokens until then
+    assert 0 < n_stopped
+    assert not any(stop for step in hist_s for _, stop, _, _ in step)
