@@ -58,6 +58,12 @@ extern "C" {
 #define ESPO_SAMPLER_FLAT  0
 #define ESPO_SAMPLER_HIER  1
 
+/* ---- stop rule (espo_params.stop_mode): the method's own rule and the ablation's replacements (Sec. 6) ---- */
+#define ESPO_STOP_ESPO         0   /* z_t > beta * max(V_phi(s_t), eps)            (Eq. 11)          */
+#define ESPO_STOP_VALUE_ONLY   1   /* V_phi(s_t) < tau                             (variant D)       */
+#define ESPO_STOP_REGRET_ONLY  2   /* z_t > tau                                    (variant E)       */
+#define ESPO_STOP_RANDOM       3   /* with probability p_random on every step      (variant F)       */
+
 /* ---- per-trajectory status (espo_state_view: status[]) ------------------------------ */
 #define ESPO_ROW_ACTIVE   0
 #define ESPO_ROW_STOPPED  1   /* ESPO's rule fired (Eq. 11): failure transition            */
@@ -87,6 +93,13 @@ typedef struct espo_params {
   int32_t t_max;            /* horizon T_max (> 0)                                          */
   int32_t eos_token;        /* end-of-sequence id, or -1 for none                           */
   int32_t sampler;          /* ESPO_SAMPLER_FLAT or ESPO_SAMPLER_HIER                       */
+  int32_t stop_mode;        /* ESPO_STOP_*; every rule is gated by warmup_complete          */
+  int32_t shadow;           /* != 0: the first step at which the rule holds is recorded in   */
+                            /* t_stop, but the trajectory is not ended and stop_out stays 0  */
+                            /* (the "Original" curves of the analysis section)               */
+  float   tau;              /* threshold of ESPO_STOP_VALUE_ONLY / ESPO_STOP_REGRET_ONLY     */
+  float   p_random;         /* per-step stop probability of ESPO_STOP_RANDOM, in [0, 1]; the */
+                            /* draw is Philox level 3, index 0 of the step's stream          */
 } espo_params;
 
 /* Opaque per-rollout-batch state: for each of `capacity` trajectory slots the smoothed

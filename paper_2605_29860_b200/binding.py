@@ -19,6 +19,7 @@ ESPO_ERR_NULL, ESPO_ERR_BAD_DTYPE, ESPO_ERR_BAD_SHAPE, ESPO_ERR_ALIGN = -1, -2, 
 ESPO_ERR_CAPACITY, ESPO_ERR_CUDA, ESPO_ERR_BAD_PARAM = -5, -6, -7
 ESPO_F32, ESPO_BF16 = 0, 1
 ESPO_SAMPLER_FLAT, ESPO_SAMPLER_HIER = 0, 1
+ESPO_STOP_ESPO, ESPO_STOP_VALUE_ONLY, ESPO_STOP_REGRET_ONLY, ESPO_STOP_RANDOM = 0, 1, 2, 3
 ESPO_ROW_ACTIVE, ESPO_ROW_STOPPED, ESPO_ROW_EOS, ESPO_ROW_TMAX, ESPO_ROW_BAD = 0, 1, 2, 3, 4
 ESPO_DEV_BAD_ROW, ESPO_DEV_BAD_SLOT, ESPO_DEV_TIMEOUT, ESPO_DEV_NAN_VALUE, ESPO_DEV_BAD_LENGTHS = 1, 2, 4, 8, 16
 
@@ -37,14 +38,16 @@ class espo_params(C.Structure):
     _fields_ = [("temperature", C.c_float), ("mu_g", C.c_float), ("sigma2_g", C.c_float),
                 ("delta", C.c_float), ("clip_c", C.c_float), ("alpha_s", C.c_float),
                 ("beta", C.c_float), ("eps", C.c_float), ("warmup_complete", C.c_int32),
-                ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32)]
+                ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32),
+                ("stop_mode", C.c_int32), ("shadow", C.c_int32), ("tau", C.c_float), ("p_random", C.c_float)]
 
 
 def make_params(temperature=1.0, mu_g=0.0, sigma2_g=1.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0,
-                eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=ESPO_SAMPLER_HIER) -> espo_params:
+                eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=ESPO_SAMPLER_HIER,
+                stop_mode=ESPO_STOP_ESPO, shadow=0, tau=0.0, p_random=0.0) -> espo_params:
     """Defaults follow the paper's hyper-parameter table (alpha_s 0.9, beta 7.0, eps 0.2, T_max 8192)."""
     return espo_params(temperature, mu_g, sigma2_g, delta, clip_c, alpha_s, beta, eps, warmup_complete, t_max,
-                       eos_token, sampler)
+                       eos_token, sampler, stop_mode, int(bool(shadow)), tau, p_random)
 
 
 _lib = None

@@ -164,6 +164,12 @@ __device__ __forceinline__ float gumbel_at(const DrawStream& ds, uint32_t level,
   return gumbel_from_word(pick_word(w, index & 3u));
 }
 
+// The uniform itself, u = (2k+1)/2^24 in (0,1).
+__device__ __forceinline__ float uniform_at(const DrawStream& ds, uint32_t level, uint32_t index) {
+  const uint4 w = philox4x32_10(index >> 2, ds.step, ds.slot, ds.batch_bits | level, ds.k0, ds.k1);
+  return __uint2float_rn(2u * (pick_word(w, index & 3u) >> 9) + 1u) * 5.9604644775390625e-08f;
+}
+
 __device__ __forceinline__ float expo_at(const DrawStream& ds, uint32_t level, uint32_t index) {
   const uint4 w = philox4x32_10(index >> 2, ds.step, ds.slot, ds.batch_bits | level, ds.k0, ds.k1);
   return expo_from_word(pick_word(w, index & 3u));

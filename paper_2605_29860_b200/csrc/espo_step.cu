@@ -72,6 +72,8 @@ struct StepArgs {
   int greedy;
   float mu_g, inv_sigma, clip_c, alpha_s, one_minus_alpha, beta, eps;
   int warmup_complete, t_max, eos_token;
+  int stop_mode, shadow;
+  float tau, p_random;
   uint32_t key0, key1, batch_bits;
   // outputs
   int32_t* tokens_out;
@@ -445,7 +447,12 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
     const bool v_nan = (v != v);
     if (v_nan) atomicOr(a.dev_status, ESPO_DEV_NAN_VALUE);
     const float thr = a.beta * fmaxf(v, a.eps);
-    const bool fires = a.warmup_complete && !v_nan && (z > thr);
+    bool rule;
+    if (a.stop_mode == ESPO_STOP_ESPO) rule = !v_nan && (z > thr);                 // Eq. 11
+    else if (a.stop_mode == ESPO_STOP_VALUE_ONLY) rule = !v_nan && (v < a.tau);
+    else if (a.stop_mode == ESPO_STOP_REGRET_ONLY) rule = (z > a.tau);
+    else rule = (uniform_at(ds, 3u, 0u) < a.p_random);
+    const bool fires = a.warmup_complete && rule;
 
     a.z[slot] = z;
     a.g[slot] = g;
@@ -458,6 +465,9 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
     uint8_t stop = 0;
     if (a.eos_token >= 0 && token == a.eos_token) {
       a.status[slot] = ESPO_ROW_EOS;
+    } else if (fires && a.shadow) {
+      if (a.t_stop[slot] < 0) a.t_stop[slot] = t_now;        // remembered, not acted upon
+      if (t_new >= a.t_max) a.status[slot] = ESPO_ROW_TMAX;
     } else if (fires) {
       a.status[slot] = ESPO_ROW_STOPPED;
       a.t_stop[slot] = t_now;
@@ -999,6 +1009,9 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   if (!(p->alpha_s >= 0.f && p->alpha_s < 1.f) || p->t_max < 1) return ESPO_ERR_BAD_PARAM;
   if (p->sampler != ESPO_SAMPLER_FLAT && p->sampler != ESPO_SAMPLER_HIER) return ESPO_ERR_BAD_PARAM;
   if (isnan(p->mu_g) || isnan(p->beta) || isnan(p->eps)) return ESPO_ERR_BAD_PARAM;
+  if (p->stop_mode < ESPO_STOP_ESPO || p->stop_mode > ESPO_STOP_RANDOM || isnan(p->tau) ||
+      !(p->p_random >= 0.f && p->p_random <= 1.f))
+    return ESPO_ERR_BAD_PARAM;
   if (n_rows == 0) return ESPO_OK;
   if (!logits || !values || !tokens_out || !stop_out) return ESPO_ERR_NULL;
   if (row_stride < st->V) return ESPO_ERR_BAD_SHAPE;
@@ -1076,6 +1089,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   a.one_minus_alpha = 1.0f - p->alpha_s;
   a.beta = p->beta; a.eps = p->eps;
   a.warmup_complete = p->warmup_complete; a.t_max = p->t_max; a.eos_token = p->eos_token;
+  a.stop_mode = p->stop_mode; a.shadow = p->shadow != 0; a.tau = p->tau; a.p_random = p->p_random;
   a.key0 = (uint32_t)(st->seed & 0xffffffffull);
   a.key1 = (uint32_t)(st->seed >> 32);
   a.batch_bits = (uint32_t)(st->batch_id << 2);

@@ -238,6 +238,38 @@ def test_compaction_and_shrinking_active_set():
     run.close()
 
 
+@pytest.mark.parametrize("mode_kw", [dict(stop_mode=espo.ESPO_STOP_VALUE_ONLY, tau=0.3),
+                                     dict(stop_mode=espo.ESPO_STOP_REGRET_ONLY, tau=0.35),
+                                     dict(stop_mode=espo.ESPO_STOP_RANDOM, p_random=0.2),
+                                     dict(stop_mode=espo.ESPO_STOP_ESPO, shadow=1),
+                                     dict(stop_mode=espo.ESPO_STOP_RANDOM, p_random=0.3, shadow=1, warmup_complete=0)])
+def test_ablation_stop_rules_and_shadow_mode(mode_kw):
+    # the replacements of Eq. 11 studied in the ablation (value only, regret only, random) and the shadow mode
+    B, V, T = 24, 5000, 10
+    kw = dict(temperature=1.0, mu_g=0.5, sigma2_g=1.0, alpha_s=0.6, beta=1.0, eps=0.2)
+    kw.update(mode_kw)
+    p = espo.make_params(**kw)
+    run = ParityRun(B, V, p, seed=33)
+    for t in range(T):
+        x = synth.logits_batch(B, V, dtype=torch.float32, sd=2.5, seed=900 + t)
+        vals = torch.rand(B, device="cuda", generator=torch.Generator("cuda").manual_seed(70 + t))
+        run.step(x, vals)
+    st = run.stats
+    t_stop = run.view["t_stop"].cpu().numpy()
+    status = run.view["status"].cpu().numpy()
+    if mode_kw.get("warmup_complete", 1) == 0:
+        assert st.stops == 0 and (t_stop == -1).all()
+    elif mode_kw.get("shadow"):
+        assert st.stops == 0 and (status == espo.ESPO_ROW_ACTIVE).all() and (t_stop >= 0).any()
+    else:
+        assert st.stops > 0 and (status == espo.ESPO_ROW_STOPPED).sum() == st.stops
+    bad = espo.make_params(stop_mode=9)
+    with pytest.raises(espo.EspoError) as e:
+        espo.espo_step(x, vals, run.state, bad, run.tokens, run.stop)
+    assert e.value.code == espo.ESPO_ERR_BAD_PARAM
+    run.close()
+
+
 def test_end_batch_updates_statistics_and_beta_like_the_oracle():
     # a short rollout in which some rows stop, then the batch-boundary update (Eq. 7-8, 12) on both sides
     B, V, T = 40, 6000, 10
