@@ -214,6 +214,15 @@ int espo_advantages(const float* rewards, const float* values, const int32_t* le
                     const uint8_t* stopped, int32_t B, int64_t total_tokens,
                     float gamma, float lambda, float r_fail, float* adv_out, void* stream);
 
+/* espo_advantages that also writes the value targets of the critic, returns_t = A_t + V(s_t) (the
+ * lambda-return that goes with the GAE of Eq. 5), in the same pass.
+ *   returns_out  device float32 [total_tokens], 16-byte aligned, or NULL (then exactly espo_advantages)
+ * Everything else as for espo_advantages. */
+int espo_advantages_returns(const float* rewards, const float* values, const int32_t* lengths,
+                            const uint8_t* stopped, int32_t B, int64_t total_tokens,
+                            float gamma, float lambda, float r_fail, float* adv_out,
+                            float* returns_out, void* stream);
+
 /* Pre-size the advantage workspace of the current device so that later calls with
  * B <= max_B and total_tokens <= max_tokens allocate nothing. */
 int espo_advantages_reserve(int32_t max_B, int64_t max_tokens);

@@ -50,6 +50,7 @@ struct AdvArgs {
   const int32_t* lengths;
   const uint8_t* stopped;
   float* adv;
+  float* ret;             // optional: returns A_t + V_t (value targets), same layout as adv; may be null
   int B;
   long long total;
   int nchunks;
@@ -320,9 +321,21 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
 #pragma unroll
       for (int h = 0; h < kAdvPerThread / 4; ++h)
         __stcs(reinterpret_cast<float4*>(a.adv + p0 + q0) + h, make_float4(out[4 * h], out[4 * h + 1], out[4 * h + 2], out[4 * h + 3]));
+      if (a.ret) {   // the values were read a moment ago: this re-read is served by L2
+#pragma unroll
+        for (int h = 0; h < kAdvPerThread / 4; ++h) {
+          const float4 vv = __ldcs(reinterpret_cast<const float4*>(a.values + p0 + q0) + h);
+          __stcs(reinterpret_cast<float4*>(a.ret + p0 + q0) + h,
+                 make_float4(out[4 * h] + vv.x, out[4 * h + 1] + vv.y, out[4 * h + 2] + vv.z, out[4 * h + 3] + vv.w));
+        }
+      }
     } else {
 #pragma unroll
-      for (int e = 0; e < kAdvPerThread; ++e) if (e < n_in) a.adv[p0 + q0 + e] = out[e];
+      for (int e = 0; e < kAdvPerThread; ++e)
+        if (e < n_in) {
+          a.adv[p0 + q0 + e] = out[e];
+          if (a.ret) a.ret[p0 + q0 + e] = out[e] + __ldcs(a.values + p0 + q0 + e);
+        }
     }
     __syncthreads();   // the next chunk's flags and carry are in place
   }
@@ -442,7 +455,7 @@ int espo_advantages_noalloc(const float* rewards, const float* values, const int
   // The array keeps whatever the previous call left.  Nothing in it has to start at zero: the preparation
   // kernel rewrites every offset and chunk owner this call reads, and the built-in status word is only OR-ed into.
   AdvArgs a;
-  a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out;
+  a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = nullptr;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
   a.gamma = (double)gamma; a.gl = (double)gamma * (double)lambda;
   a.r_fail = r_fail;
@@ -462,14 +475,15 @@ int espo_advantages_reserve(int32_t max_B, int64_t max_tokens) {
   return ensure_pool(dev, max_B, (max_tokens + kAdvChunk - 1) / kAdvChunk, &p);
 }
 
-int espo_advantages(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
-                    int32_t B, int64_t total_tokens, float gamma, float lambda, float r_fail, float* adv_out,
-                    void* stream) {
+int espo_advantages_returns(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
+                            int32_t B, int64_t total_tokens, float gamma, float lambda, float r_fail, float* adv_out,
+                            float* returns_out, void* stream) {
   using namespace espo;
   if (B < 0 || total_tokens < 0) return ESPO_ERR_BAD_SHAPE;
   if (B == 0 || total_tokens == 0) return ESPO_OK;
   if (!rewards || !values || !lengths || !stopped || !adv_out) return ESPO_ERR_NULL;
-  if (((uintptr_t)rewards % 16) || ((uintptr_t)values % 16) || ((uintptr_t)adv_out % 16) || ((uintptr_t)lengths % 4))
+  if (((uintptr_t)rewards % 16) || ((uintptr_t)values % 16) || ((uintptr_t)adv_out % 16) || ((uintptr_t)lengths % 4) ||
+      ((uintptr_t)returns_out % 16))
     return ESPO_ERR_ALIGN;
   if (gamma != gamma || lambda != lambda || r_fail != r_fail) return ESPO_ERR_BAD_PARAM;
   const long long nchunks = (total_tokens + kAdvChunk - 1) / kAdvChunk;
@@ -482,12 +496,19 @@ int espo_advantages(const float* rewards, const float* values, const int32_t* le
   if (rc != ESPO_OK) return rc;
   cudaStream_t s = (cudaStream_t)stream;
   AdvArgs a;
-  a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out;
+  a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = returns_out;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
   a.gamma = (double)gamma; a.gl = (double)gamma * (double)lambda;
   a.r_fail = r_fail;
   a.ws = p->ws;
   return launch_advantages(a, p->sm_count, s);
+}
+
+int espo_advantages(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
+                    int32_t B, int64_t total_tokens, float gamma, float lambda, float r_fail, float* adv_out,
+                    void* stream) {
+  return espo_advantages_returns(rewards, values, lengths, stopped, B, total_tokens, gamma, lambda, r_fail, adv_out,
+                                 nullptr, stream);
 }
 
 int espo_advantages_status(uint32_t* host_out, void* stream) {

@@ -83,3 +83,27 @@ def test_reserve_then_smaller_calls():
     for seed in (5, 6):
         r, v, L, s = synth.ragged_trajectories(300, len_lo=1, len_hi=3000, seed=seed)
         _check(r, v, L, s, 1.0, 0.95, -1.0)
+
+
+def test_returns_are_written_in_the_same_pass():
+    # value targets A_t + V_t; with gamma = lambda = 1 they are the reward-to-go with the failure transition applied
+    r, v, L, s = synth.ragged_trajectories(300, len_lo=1, len_hi=9000, seed=8)
+    adv, ret = torch.empty_like(r), torch.empty_like(r)
+    for gamma, lam in ((1.0, 1.0), (0.99, 0.95)):
+        espo.espo_advantages_returns(r, v, L, s, gamma, lam, -1.0, adv, ret)
+        torch.cuda.synchronize()
+        ref = oracle.advantages(r.cpu().numpy(), v.cpu().numpy(), L.cpu().numpy(), s.cpu().numpy(), gamma, lam, -1.0)
+        want = ref + v.cpu().numpy().astype(np.float64)
+        got = ret.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - want) <= 2e-5 + 1e-4 * np.abs(want))
+        assert np.all(np.abs(adv.cpu().numpy() - ref) <= 1e-5 + 1e-4 * np.abs(ref))
+        if gamma == 1.0 and lam == 1.0:
+            rr = r.cpu().numpy().astype(np.float64)
+            off = np.concatenate([[0], np.cumsum(L.cpu().numpy().astype(np.int64))])
+            for i in (0, 7, 150, 299):
+                seg = rr[off[i]:off[i + 1]].copy()
+                if seg.size and s[i]:
+                    seg[-1] = -1.0
+                togo = np.cumsum(seg[::-1])[::-1]
+                assert np.allclose(got[off[i]:off[i + 1]], togo, rtol=1e-4, atol=2e-5)
+    assert espo.espo_advantages_status() == 0
