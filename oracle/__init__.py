@@ -59,7 +59,7 @@ class RowState(C.Structure):
 class StepOut(C.Structure):
     _fields_ = [("g", C.c_double), ("g_tilde", C.c_double), ("z", C.c_double), ("logp", C.c_double),
                 ("max_x", C.c_double), ("log_s", C.c_double), ("min_rel_gap", C.c_double),
-                ("threshold", C.c_double), ("token", C.c_int32), ("stop", C.c_int32),
+                ("threshold", C.c_double), ("entropy", C.c_double), ("token", C.c_int32), ("stop", C.c_int32),
                 ("runner_up", C.c_int32), ("bad", C.c_int32)]
 
 

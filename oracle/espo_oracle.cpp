@@ -180,6 +180,7 @@ struct espo_oracle_step_out {
   double max_x, log_s;           // max_a x_a and log sum_a exp(x_a - max_x)
   double min_rel_gap;            // smallest top-two relative gap over the argmaxes taken
   double threshold;              // beta * max(V, eps)
+  double entropy;                // H(pi(.|s_t)) = -sum_a pi(a) log pi(a), the quantity tracked in the analysis section
   int32_t token;
   int32_t stop;
   int32_t runner_up;             // token that the closest argmax would have produced instead (-1 unknown)
@@ -251,6 +252,15 @@ void espo_oracle_step_row(const double* logits, int64_t V, double value,
   for (int64_t a = 0; a < V; ++a) s += std::exp(x[a] - m);
   out->max_x = m;
   out->log_s = std::log(s);
+  {
+    // entropy of the sampling distribution, term by term (0 log 0 = 0 for masked ids)
+    double h = 0.0;
+    for (int64_t a = 0; a < V; ++a) {
+      const double lp = x[a] - m - out->log_s;
+      if (lp > NEG_INF) h -= std::exp(lp) * lp;
+    }
+    out->entropy = greedy ? 0.0 : h;
+  }
 
   const DrawKey dk{seed, batch_id, slot, (uint32_t)st->t};
   int64_t token = -1;

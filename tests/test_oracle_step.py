@@ -447,3 +447,19 @@ def test_shadow_mode_records_the_first_firing_step_and_keeps_decoding():
         assert [h[r][0] for h in hist_s[:upto]] == [h[r][0] for h in hist_a[:upto]]   # same tokens until then
     assert 0 < n_stopped
     assert not any(stop for step in hist_s for _, stop, _, _ in step)
+
+
+# --------------------------------------------------------------------------- policy entropy (analysis section)
+
+
+def test_entropy_matches_library_and_closed_forms():
+    rng = _rng(60)
+    V = 700
+    x = _peaked_logits(rng, 3, V)
+    x[1, :] = 1.25                      # uniform: H = log V
+    x[2, :] = -np.inf; x[2, 5] = 0.0    # one admissible id: H = 0
+    for T in (1.0, 0.6):
+        outs = oracle.Rollout(3, seed=2).step(x, np.zeros(3), oracle.make_params(temperature=T, warmup_complete=0))
+        assert abs(outs[0].entropy - stats.entropy(special.softmax(x[0] / T))) < 1e-10
+        assert abs(outs[1].entropy - math.log(V)) < 1e-10
+        assert outs[2].entropy == 0.0 and outs[2].token == 5
