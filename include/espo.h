@@ -100,6 +100,9 @@ typedef struct espo_params {
   float   tau;              /* threshold of ESPO_STOP_VALUE_ONLY / ESPO_STOP_REGRET_ONLY     */
   float   p_random;         /* per-step stop probability of ESPO_STOP_RANDOM, in [0, 1]; the */
                             /* draw is Philox level 3, index 0 of the step's stream          */
+  int32_t want_entropy;     /* != 0: also compute the policy entropy H(pi(.|s_t)) in the same */
+                            /* pass (the quantity tracked in the analysis section); needs    */
+                            /* ESPO_SAMPLER_HIER                                              */
 } espo_params;
 
 /* Opaque per-rollout-batch state: for each of `capacity` trajectory slots the smoothed
@@ -156,10 +159,13 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride,
  * pointer may be NULL.  g, g_tilde and logp hold the values of each slot's latest step
  * (logp = log pi(a_t | s_t) under the temperature-scaled distribution).  t is the number
  * of tokens generated; t_stop is the index of the stop step or -1; sum_g, sum_g2 are the
- * double-precision sums over the slot's tokens that the batch statistics of Eq. 7-8 need. */
+ * double-precision sums over the slot's tokens that the batch statistics of Eq. 7-8 need;
+ * entropy is the policy entropy of the slot's latest step and sum_h its running sum (both only
+ * maintained by steps with want_entropy set). */
 int espo_state_view(espo_state* st, const float** z, const float** g, const float** g_tilde,
                     const float** logp, const int32_t** t, const uint8_t** status,
-                    const int32_t** t_stop, const double** sum_g, const double** sum_g2);
+                    const int32_t** t_stop, const double** sum_g, const double** sum_g2,
+                    const float** entropy, const double** sum_h);
 
 /* Expert knob: override the step kernel's launch shape for this state.  consumer_warps =
  * streaming warps per CTA (1..31), stages = blocks of 1024 ids each warp keeps in flight,

@@ -39,15 +39,16 @@ class espo_params(C.Structure):
                 ("delta", C.c_float), ("clip_c", C.c_float), ("alpha_s", C.c_float),
                 ("beta", C.c_float), ("eps", C.c_float), ("warmup_complete", C.c_int32),
                 ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32),
-                ("stop_mode", C.c_int32), ("shadow", C.c_int32), ("tau", C.c_float), ("p_random", C.c_float)]
+                ("stop_mode", C.c_int32), ("shadow", C.c_int32), ("tau", C.c_float), ("p_random", C.c_float),
+                ("want_entropy", C.c_int32)]
 
 
 def make_params(temperature=1.0, mu_g=0.0, sigma2_g=1.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0,
                 eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=ESPO_SAMPLER_HIER,
-                stop_mode=ESPO_STOP_ESPO, shadow=0, tau=0.0, p_random=0.0) -> espo_params:
+                stop_mode=ESPO_STOP_ESPO, shadow=0, tau=0.0, p_random=0.0, want_entropy=0) -> espo_params:
     """Defaults follow the paper's hyper-parameter table (alpha_s 0.9, beta 7.0, eps 0.2, T_max 8192)."""
     return espo_params(temperature, mu_g, sigma2_g, delta, clip_c, alpha_s, beta, eps, warmup_complete, t_max,
-                       eos_token, sampler, stop_mode, int(bool(shadow)), tau, p_random)
+                       eos_token, sampler, stop_mode, int(bool(shadow)), tau, p_random, int(bool(want_entropy)))
 
 
 _lib = None
@@ -70,7 +71,7 @@ def lib():
         L.espo_free_state.restype = None
         L.espo_set_launch_config.argtypes = [vp, i32, i32, i32]
         L.espo_step.argtypes = [vp, i32, i64, vp, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp, vp]
-        L.espo_state_view.argtypes = [vp] + [C.POINTER(vp)] * 9
+        L.espo_state_view.argtypes = [vp] + [C.POINTER(vp)] * 11
         L.espo_compact_active.argtypes = [vp, vp, vp, vp]
         L.espo_state_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.espo_end_batch.argtypes = [vp, f32, f32, f32, f32, f32, i32, C.POINTER(espo_params), C.POINTER(C.c_double), vp]
@@ -191,10 +192,10 @@ class _DevArray:
 
 def espo_state_view(state: EspoState) -> dict:
     """Torch views (treat as read-only) of the per-slot arrays: z, g, g_tilde, logp, t, status, t_stop, sum_g, sum_g2."""
-    ptrs = [C.c_void_p() for _ in range(9)]
+    ptrs = [C.c_void_p() for _ in range(11)]
     _check(lib().espo_state_view(state.handle, *[C.byref(p) for p in ptrs]), "espo_state_view")
-    names = ["z", "g", "g_tilde", "logp", "t", "status", "t_stop", "sum_g", "sum_g2"]
-    types = ["<f4", "<f4", "<f4", "<f4", "<i4", "|u1", "<i4", "<f8", "<f8"]
+    names = ["z", "g", "g_tilde", "logp", "t", "status", "t_stop", "sum_g", "sum_g2", "entropy", "sum_h"]
+    types = ["<f4", "<f4", "<f4", "<f4", "<i4", "|u1", "<i4", "<f8", "<f8", "<f4", "<f8"]
     with torch.cuda.device(state.device):
         return {n: torch.as_tensor(_DevArray(p.value, state.capacity, ty), device=state.device)
                 for n, p, ty in zip(names, ptrs, types)}

@@ -62,6 +62,8 @@ struct StepArgs {
   int32_t *t, *t_stop;
   uint8_t* status;
   double *sum_g, *sum_g2;
+  float* entropy;       // per slot: H(pi(.|s_t)) of the latest step (only written when want_entropy)
+  double* sum_h;        // per slot: running sum of those
   // scratch (indexed by row of this call)
   float4* records;      // [capacity * nblk] block records
   unsigned* ticket;     // [capacity] blocks of the row reduced so far
@@ -72,7 +74,7 @@ struct StepArgs {
   int greedy;
   float mu_g, inv_sigma, clip_c, alpha_s, one_minus_alpha, beta, eps;
   int warmup_complete, t_max, eos_token;
-  int stop_mode, shadow;
+  int stop_mode, shadow, want_entropy;
   float tau, p_random;
   uint32_t key0, key1, batch_bits;
   // outputs
@@ -188,11 +190,26 @@ __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned c
   const float c0 = -ref * a.k2;
   const float2 c0v = make_float2(c0, c0);
   float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+  float u_b = 0.f;   // sum of e * t with t = (x - ref) k2 <= 0, e = 2^t: what the entropy needs besides the sum of e
+  if (SAMPLER == ESPO_SAMPLER_HIER && a.want_entropy) {
+    float2 ua = make_float2(0.f, 0.f);
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    const float2 t = __ffma2_rn(bv.pair(j), k2v, c0v);
-    const float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
-    if (j & 1) acc1 = __fadd2_rn(acc1, e); else acc0 = __fadd2_rn(acc0, e);
+    for (int j = 0; j < 16; ++j) {
+      float2 t = __ffma2_rn(bv.pair(j), k2v, c0v);
+      const float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
+      if (e.x == 0.f) t.x = 0.f;   // masked ids (t = -inf): 0 * -inf is not a number
+      if (e.y == 0.f) t.y = 0.f;
+      ua = __ffma2_rn(e, t, ua);
+      if (j & 1) acc1 = __fadd2_rn(acc1, e); else acc0 = __fadd2_rn(acc0, e);
+    }
+    u_b = warp_sum(ua.x + ua.y);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float2 t = __ffma2_rn(bv.pair(j), k2v, c0v);
+      const float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
+      if (j & 1) acc1 = __fadd2_rn(acc1, e); else acc0 = __fadd2_rn(acc0, e);
+    }
   }
   const float s_b = warp_sum((acc0.x + acc0.y) + (acc1.x + acc1.y));
 
@@ -214,7 +231,7 @@ __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned c
     warp_argmax(best, best_id);
     if (lane == 0) static_cast<float4*>(rec_row)[block] = make_float4(m_b, s_b, best, __int_as_float(best_id));
   } else {
-    if (lane == 0) static_cast<float4*>(rec_row)[block] = make_float4(m_b, s_b, 0.f, 0.f);
+    if (lane == 0) static_cast<float4*>(rec_row)[block] = make_float4(m_b, s_b, u_b, 0.f);
   }
 }
 
@@ -303,7 +320,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
   float best = NINF;          // best perturbed score among this lane's blocks (greedy: largest block maximum)
   int best_i = -1;            // HIER / greedy: block number; FLAT: token id
   bool poisoned = false;
-  float run_m = NINF, run_s = 0.f;
+  float run_m = NINF, run_s = 0.f, run_u = 0.f;   // sums of e and of e*t over this lane's blocks, relative to run_m
   auto load_rec = [&](int b) -> float4 {
     const float4* rp = static_cast<const float4*>(rec_row) + b;
     return rec_local ? *rp : __ldcg(rp);       // shared-memory table, or global records written by other CTAs
@@ -337,20 +354,39 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       poisoned |= !(r[i].y >= 0.0f) || isinf(r[i].y);   // NaN or inf sum: the block held NaN or +inf
       if (r[i].y > 0.f) lm = fmaxf(lm, r[i].x);
     }
-    // sum of s_b 2^((m_b - lm) k2), independent terms; the carried sum is rescaled once
-    float acc = (run_m == lm) ? run_s : run_s * ex2_approx((run_m - lm) * a.k2);
+    // sum of s_b 2^((m_b - lm) k2), independent terms; the carried sums are rescaled once.  Moving the reference
+    // from R to R' turns (S, U) into f (S, U + (R - R') k2 S) with f = 2^((R - R') k2).
+    float acc = run_s, accu = run_u;
+    if (run_m != lm && run_s > 0.f) {
+      const float dt = (run_m - lm) * a.k2, f = ex2_approx(dt);
+      accu = f * fmaf(dt, run_s, run_u);
+      acc = f * run_s;
+    }
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i)
-      if (r[i].y > 0.f) acc = fmaf(r[i].y, ex2_approx((r[i].x - lm) * a.k2), acc);
-    run_m = lm; run_s = acc;
+      if (r[i].y > 0.f) {
+        const float dt = (r[i].x - lm) * a.k2, f = ex2_approx(dt);
+        acc = fmaf(r[i].y, f, acc);
+        if (SAMPLER == ESPO_SAMPLER_HIER) accu = fmaf(f, fmaf(dt, r[i].y, r[i].z), accu);
+      }
+    run_m = lm; run_s = acc; run_u = accu;
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i) score(base + 32 * i + lane, r[i]);
   }
   {
     const float mm = warp_max(run_m);
-    if (run_m != mm) run_s *= ex2_approx((run_m - mm) * a.k2);   // run_m = -inf: run_s is 0 and stays 0
+    if (run_m != mm) {
+      if (run_s > 0.f) {
+        const float dt = (run_m - mm) * a.k2, f = ex2_approx(dt);
+        run_u = f * fmaf(dt, run_s, run_u);
+        run_s *= f;
+      } else {
+        run_s = 0.f; run_u = 0.f;     // a lane without blocks (run_m = -inf)
+      }
+    }
     run_m = mm;
     run_s = warp_sum(run_s);
+    run_u = warp_sum(run_u);
   }
   const float M = run_m, S = run_s;
   const float log_S = logf(S);   // needed at the very end; started before the loads below
@@ -460,6 +496,12 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
     a.logp[slot] = logp;
     a.sum_g[slot] = pre.sum_g + (double)g;
     a.sum_g2[slot] = pre.sum_g2 + (double)g * (double)g;
+    if (a.want_entropy) {
+      // H = ln S - ln2 * U / S with S, U the sums of e and of e*t relative to the row maximum
+      const float h = a.greedy ? 0.f : fmaxf(log_S - 0.6931471805599453f * run_u / S, 0.f);
+      a.entropy[slot] = h;
+      a.sum_h[slot] += (double)h;
+    }
     const int t_new = t_now + 1;
     a.t[slot] = t_new;
     uint8_t stop = 0;
@@ -806,6 +848,8 @@ struct espo_state {
   int32_t *t, *t_stop;
   uint8_t* status;
   double *sum_g, *sum_g2;
+  float* entropy;
+  double* sum_h;
   float4* records;
   unsigned *ticket, *dev_status;
   double* batch_out;   // [8] result of espo_end_batch
@@ -944,7 +988,7 @@ int espo_init_state(espo_state** out, int32_t capacity, int32_t V, uint64_t seed
   auto carve = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const size_t o_z = carve(4 * cap), o_g = carve(4 * cap), o_gt = carve(4 * cap), o_lp = carve(4 * cap);
   const size_t o_t = carve(4 * cap), o_ts = carve(4 * cap), o_st = carve(cap);
-  const size_t o_sg = carve(8 * cap), o_sg2 = carve(8 * cap);
+  const size_t o_sg = carve(8 * cap), o_sg2 = carve(8 * cap), o_h = carve(4 * cap), o_sh = carve(8 * cap);
   const size_t o_rec = carve(sizeof(float4) * cap * (size_t)st->nblk);
   const size_t o_tk = carve(4 * cap), o_ds = carve(4), o_bo = carve(8 * 8);
   st->arena_bytes = off;
@@ -954,6 +998,7 @@ int espo_init_state(espo_state** out, int32_t capacity, int32_t V, uint64_t seed
   st->z = (float*)(base + o_z); st->g = (float*)(base + o_g); st->g_tilde = (float*)(base + o_gt);
   st->logp = (float*)(base + o_lp); st->t = (int32_t*)(base + o_t); st->t_stop = (int32_t*)(base + o_ts);
   st->status = (uint8_t*)(base + o_st); st->sum_g = (double*)(base + o_sg); st->sum_g2 = (double*)(base + o_sg2);
+  st->entropy = (float*)(base + o_h); st->sum_h = (double*)(base + o_sh);
   st->records = (float4*)(base + o_rec); st->ticket = (unsigned*)(base + o_tk); st->dev_status = (unsigned*)(base + o_ds);
   st->batch_out = (double*)(base + o_bo);
 
@@ -1012,6 +1057,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   if (p->stop_mode < ESPO_STOP_ESPO || p->stop_mode > ESPO_STOP_RANDOM || isnan(p->tau) ||
       !(p->p_random >= 0.f && p->p_random <= 1.f))
     return ESPO_ERR_BAD_PARAM;
+  if (p->want_entropy && p->sampler != ESPO_SAMPLER_HIER) return ESPO_ERR_BAD_PARAM;   // the flat sampler's records are full
   if (n_rows == 0) return ESPO_OK;
   if (!logits || !values || !tokens_out || !stop_out) return ESPO_ERR_NULL;
   if (row_stride < st->V) return ESPO_ERR_BAD_SHAPE;
@@ -1075,7 +1121,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   if (smem > (size_t)st->max_smem) return ESPO_ERR_CAPACITY;
 
   a.z = st->z; a.g = st->g; a.g_tilde = st->g_tilde; a.logp = st->logp;
-  a.t = st->t; a.t_stop = st->t_stop; a.status = st->status; a.sum_g = st->sum_g; a.sum_g2 = st->sum_g2;
+  a.t = st->t; a.t_stop = st->t_stop; a.status = st->status; a.sum_g = st->sum_g; a.sum_g2 = st->sum_g2; a.entropy = st->entropy; a.sum_h = st->sum_h;
   a.records = st->records; a.ticket = st->ticket; a.dev_status = st->dev_status;
 
   a.greedy = (p->temperature == 0.f);
@@ -1089,6 +1135,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   a.one_minus_alpha = 1.0f - p->alpha_s;
   a.beta = p->beta; a.eps = p->eps;
   a.warmup_complete = p->warmup_complete; a.t_max = p->t_max; a.eos_token = p->eos_token;
+  a.want_entropy = p->want_entropy != 0;
   a.stop_mode = p->stop_mode; a.shadow = p->shadow != 0; a.tau = p->tau; a.p_random = p->p_random;
   a.key0 = (uint32_t)(st->seed & 0xffffffffull);
   a.key1 = (uint32_t)(st->seed >> 32);
@@ -1104,7 +1151,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
 
 int espo_state_view(espo_state* st, const float** z, const float** g, const float** g_tilde, const float** logp,
                     const int32_t** t, const uint8_t** status, const int32_t** t_stop, const double** sum_g,
-                    const double** sum_g2) {
+                    const double** sum_g2, const float** entropy, const double** sum_h) {
   if (!st) return ESPO_ERR_NULL;
   if (z) *z = st->z;
   if (g) *g = st->g;
@@ -1115,6 +1162,8 @@ int espo_state_view(espo_state* st, const float** z, const float** g, const floa
   if (t_stop) *t_stop = st->t_stop;
   if (sum_g) *sum_g = st->sum_g;
   if (sum_g2) *sum_g2 = st->sum_g2;
+  if (entropy) *entropy = st->entropy;
+  if (sum_h) *sum_h = st->sum_h;
   return ESPO_OK;
 }
 

@@ -64,6 +64,7 @@ class ParityRun:
         # slots the oracle follows (rows are independent, so a subset is a valid check)
         self.check = set(range(capacity)) if check_slots is None else set(int(s) for s in check_slots)
         self.dropped = set()
+        self.entropy_log = {}      # slot -> oracle entropies of its steps (when params.want_entropy)
 
     def step(self, logits: torch.Tensor, values: torch.Tensor, row_ids: torch.Tensor | None = None):
         n = logits.shape[0]
@@ -104,6 +105,10 @@ class ParityRun:
                 got = float(v[name][s])
                 assert close(got, ref), f"row {r} slot {s} t={before[i].t}: {name} gpu={got!r} oracle={ref!r}"
                 self.stats.max_err = max(self.stats.max_err, abs(got - ref))
+            if self.params.want_entropy:
+                got = float(v["entropy"][s])
+                assert close(got, o.entropy), f"row {r} slot {s} t={before[i].t}: entropy gpu={got!r} oracle={o.entropy!r}"
+                self.entropy_log.setdefault(s, []).append(o.entropy)
             ost = self.ro.states[s]
             if int(stp[r]) != o.stop or int(v["status"][s]) != ost.status:
                 margin = abs(o.z - o.threshold)

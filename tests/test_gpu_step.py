@@ -270,6 +270,31 @@ def test_ablation_stop_rules_and_shadow_mode(mode_kw):
     run.close()
 
 
+@pytest.mark.parametrize("V,dtype,temperature", [(152064, torch.bfloat16, 1.0), (152064, torch.bfloat16, 0.6),
+                                                   (5000, torch.float32, 1.3), (1025, torch.bfloat16, 1.0)])
+def test_policy_entropy_in_the_same_pass(V, dtype, temperature):
+    B, T = 6, 3
+    p = espo.make_params(temperature=temperature, mu_g=1.0, sigma2_g=2.0, beta=50.0, want_entropy=1)
+    run = ParityRun(B, V, p, seed=17)
+    for t in range(T):
+        x = synth.logits_batch(B, V, dtype=dtype, sd=3.0 if t else 0.5, seed=40 + t)   # flat rows, then peaked ones
+        if t == 1:
+            x[0, : V // 2] = float("-inf")        # masked ids contribute nothing
+        run.step(x, torch.full((B,), 0.5, device="cuda"))
+    h = run.view["entropy"].cpu().numpy()
+    assert (h >= 0).all() and (h <= np.log(V) + 1e-4).all()
+    assert abs(float(run.view["sum_h"][1]) - sum_h_of(run, 1)) < 1e-3
+    with pytest.raises(espo.EspoError) as e:
+        espo.espo_step(x, torch.zeros(B, device="cuda"), run.state,
+                       espo.make_params(want_entropy=1, sampler=espo.ESPO_SAMPLER_FLAT), run.tokens, run.stop)
+    assert e.value.code == espo.ESPO_ERR_BAD_PARAM
+    run.close()
+
+
+def sum_h_of(run, slot):
+    return float(sum(run.entropy_log[slot]))
+
+
 def test_end_batch_updates_statistics_and_beta_like_the_oracle():
     # a short rollout in which some rows stop, then the batch-boundary update (Eq. 7-8, 12) on both sides
     B, V, T = 40, 6000, 10
