@@ -192,7 +192,7 @@ def main():
     import numpy as np
     import torch
     import paper_2605_29860_b200 as espo
-    from paper_2605_29860_b200 import synth
+    from paper_2605_29860_b200 import shard, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -210,12 +210,13 @@ def main():
     sampler = espo.ESPO_SAMPLER_HIER if args.sampler == "hier" else espo.ESPO_SAMPLER_FLAT
     params = espo.make_params(sampler=sampler, **PARAMS)
     # ---- synthetic inputs, resident in HBM: every rank owns its own B rows (rows are independent) ----
-    bufs = [synth.logits_batch(B, V, dtype=torch.bfloat16, sd=3.0, seed=100 + 10 * rank + i, device=dev)
+    plan = shard.rank_plan(rank, world, B)
+    bufs = [synth.logits_batch(B, V, dtype=torch.bfloat16, sd=3.0, seed=100 + plan["data_seed_offset"] + i, device=dev)
             for i in range(N_BUFFERS)]
     values = torch.full((B,), 0.5, dtype=torch.bfloat16, device=dev)
     tokens = torch.empty(B, dtype=torch.int32, device=dev)
     stop = torch.empty(B, dtype=torch.uint8, device=dev)
-    state = espo.espo_init_state(B, V, seed=1234 + rank)
+    state = espo.espo_init_state(B, V, seed=plan["state_seed"])
     view = espo.espo_state_view(state)
     # rollout record for the closing advantage pass: K tokens per trajectory, reward 0 except the end
     adv_tokens = B * K
@@ -277,10 +278,7 @@ def main():
     t_wall1 = time.time()
     ms_total = ev0.elapsed_time(ev2)
     ms_steps = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_total, ms_steps], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_steps = t.tolist()
+    ms_total, ms_steps = shard.max_over_ranks([ms_total, ms_steps], dist, device=dev)
     if sampler_proc:
         time.sleep(0.1)
         sampler_proc.stop()

@@ -1,0 +1,48 @@
+"""Row sharding across GPUs for the ESPO hot path.
+
+Trajectories are independent units: neither ``espo_step`` nor ``espo_advantages`` exchanges data
+between rows, so N GPUs run N disjoint row ranges with no data-path collective.  This module holds
+the little host-side logic that goes with it: which rows and seeds a rank owns, and the reduction
+of per-rank timings (the only communication the benchmark does).
+"""
+from __future__ import annotations
+
+from typing import List, Tuple
+
+import torch
+
+
+def shard_rows(n_rows: int, world: int) -> List[Tuple[int, int]]:
+    """Contiguous, disjoint row ranges [lo, hi) that cover 0..n_rows, sizes differing by at most one."""
+    if world < 1 or n_rows < 0:
+        raise ValueError("world must be >= 1 and n_rows >= 0")
+    return [(r * n_rows // world, (r + 1) * n_rows // world) for r in range(world)]
+
+
+def rank_plan(rank: int, world: int, rows_per_rank: int, base_seed: int = 1234) -> dict:
+    """Weak-scaling plan: every rank owns ``rows_per_rank`` trajectories of one global batch.
+
+    Returns the rank's slice of global trajectory ids, the Philox seed of its state and the seed offset
+    of its synthetic inputs; both seeds differ between ranks so that no two GPUs draw the same noise.
+    """
+    if not 0 <= rank < world:
+        raise ValueError("rank outside [0, world)")
+    lo = rank * rows_per_rank
+    return {"rows": (lo, lo + rows_per_rank), "state_seed": base_seed + rank, "data_seed_offset": 10 * rank,
+            "global_rows": world * rows_per_rank}
+
+
+def max_over_ranks(values, dist=None, device="cpu") -> list:
+    """Element-wise maximum of a list of floats over all ranks (the timings of a multi-GPU run)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def sum_over_ranks(values, dist=None, device="cpu") -> list:
+    """Element-wise sum over all ranks (rows processed, rows stopped)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return t.tolist()
