@@ -55,6 +55,7 @@ struct StepArgs {
   int nblk;                 // 1024-id blocks per row
   long long total_blocks;   // n_rows * nblk
   int warps, fin_warps, stages, stage_bytes, queue_cap;   // streaming warps, finalizer warps, ring depth
+  int run_len;              // consecutive blocks a streaming warp takes per turn (1 unless rows are short)
   int local_rows;           // rows whose block records fit in the CTA's shared-memory table (0: none)
   int noise_rows;           // rows whose block-level noise fits in the CTA's shared-memory table
   // trajectory state (indexed by slot)
@@ -692,12 +693,23 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
     unsigned char* my_ring = ring + (size_t)warp * S * a.stage_bytes;
     uint64_t* my_bar = bars + warp * S;
     int2* my_meta = metas + warp * S;            // (local row, block) of the block each stage holds
-    const int n_my = (cr.n > warp) ? (cr.n - warp + W - 1) / W : 0;
+    // The warps take turns of C consecutive positions of the CTA's walk: warp w owns the runs w, w + W, w + 2W, ...
+    // (C = 1 for long rows; short rows use longer runs so that a warp reports to a row once per run, not per block).
+    const int C = a.run_len;
+    int n_my = 0;
+    {
+      const int n_runs = (cr.n + C - 1) / C;
+      if (n_runs > warp) {
+        const int mine = (n_runs - warp + W - 1) / W;            // runs owned by this warp
+        n_my = mine * C;
+        if ((n_runs - 1) % W == warp) n_my -= n_runs * C - cr.n;  // the walk's last run may be short
+      }
+    }
     constexpr int kBlockBytes = kBlockIds * ES;
 
-    // Where the warp's next block to fetch lies.  The warp takes every W-th position of the CTA's walk, so the
-    // cursor moves by W blocks at a time and only divides when the walk wraps around the end of the range.
-    int fq, f_lrow, f_blk;
+    // Where the warp's next block to fetch lies.  The cursor moves by one block inside a run and by (W-1)C+1
+    // between runs, and only divides when the walk wraps around the end of the range.
+    int fq, f_lrow, f_blk, f_run = 0;
     const unsigned char* f_ptr;
     auto seek = [&](int q) {
       fq = q;
@@ -707,10 +719,12 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
       f_ptr = a.logits + (size_t)(cr.r_first + f_lrow) * a.row_stride_bytes + (size_t)f_blk * kBlockBytes;
     };
     auto advance = [&]() {
-      fq += W;
-      if (fq >= cr.n) { seek(fq - cr.n); return; }
-      f_blk += W;
-      f_ptr += (size_t)W * kBlockBytes;
+      int step = 1;
+      if (++f_run == C) { f_run = 0; step = (W - 1) * C + 1; }
+      if (fq + step >= cr.n) { seek(fq + step - cr.n); return; }
+      fq += step;
+      f_blk += step;
+      f_ptr += (size_t)step * kBlockBytes;
       while (f_blk >= cr.nblk) {
         f_blk -= cr.nblk;
         ++f_lrow;
@@ -718,7 +732,7 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
       }
     };
     {
-      int q = warp + cr.off;
+      int q = warp * C + cr.off;
       if (q >= cr.n) q -= cr.n;
       seek(n_my > 0 ? q : 0);
     }
@@ -1116,6 +1130,7 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   if (per_warp < stages) stages = (int)per_warp;
   a.warps = warps;
   a.fin_warps = fin;
+  a.run_len = (st->nblk >= 64) ? 1 : (st->nblk >= 32 ? 4 : (st->nblk >= 8 ? 2 : 1));
   a.stages = stages;
   const size_t smem = footprint(warps, stages);
   if (smem > (size_t)st->max_smem) return ESPO_ERR_CAPACITY;
