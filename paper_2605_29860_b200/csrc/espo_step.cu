@@ -247,13 +247,13 @@ __device__ __forceinline__ float load_logit(const unsigned char* row_base, int i
 }
 
 __device__ __forceinline__ void mark_row(const StepArgs& a, int row, int slot, int lane, int32_t token, unsigned dev_bit,
-                                         int new_status, bool rec_local) {
+                                         int new_status, bool no_ticket) {
   if (lane == 0) {
     if (dev_bit) atomicOr(a.dev_status, dev_bit);
     if (new_status >= 0) a.status[slot] = (uint8_t)new_status;
     a.tokens_out[row] = token;
     a.stop_out[row] = 0;
-    a.ticket[row] = 0;   // ready for the next launch
+    if (!no_ticket) a.ticket[row] = 0;   // ready for the next launch
   }
 }
 
@@ -304,11 +304,11 @@ __device__ __forceinline__ float sum_exp2_32(const float (&x)[kSubIds], float m,
 // log-sum-exp  m/T + ln s  the score is  m/T + ln(s / E).
 template <int ES, int SAMPLER>
 __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, const RowPre pre, const void* rec_row,
-                                          bool rec_local, const float* noise) {
+                                          bool rec_local, bool no_ticket, const float* noise) {
   const float NINF = __int_as_float(0xff800000);
   const int slot = pre.slot;
-  if (slot < 0) { mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, rec_local); return; }
-  if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, slot, lane, -1, 0u, -1, rec_local); return; }   // finished: untouched
+  if (slot < 0) { mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, no_ticket); return; }
+  if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, slot, lane, -1, 0u, -1, no_ticket); return; }   // finished: untouched
   const int t_now = pre.t_now;
   const unsigned char* row_base = a.logits + (size_t)row * a.row_stride_bytes;
   const DrawStream ds{a.key0, a.key1, (uint32_t)t_now, (uint32_t)slot, a.batch_bits};
@@ -392,9 +392,9 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
   const float M = run_m, S = run_s;
   const float log_S = logf(S);   // needed at the very end; started before the loads below
   poisoned = __any_sync(kFullMask, poisoned) || !(M > NINF) || isinf(M);
-  if (poisoned) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, rec_local); return; }
+  if (poisoned) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, no_ticket); return; }
   warp_argmax(best, best_i);
-  if (best_i < 0) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, rec_local); return; }   // nothing to pick from
+  if (best_i < 0) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, no_ticket); return; }   // nothing to pick from
 
   int token;
   float l_tok;
@@ -520,7 +520,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
     }
     a.tokens_out[row] = token;
     a.stop_out[row] = stop;
-    if (!rec_local) a.ticket[row] = 0;   // ready for the next launch
+    if (!no_ticket) a.ticket[row] = 0;   // ready for the next launch
   }
 }
 
@@ -594,10 +594,19 @@ __device__ void drain_queue(const StepArgs& a, const CtaRange& cr, StepCtrl* ctr
     if (li >= 0) {
       // every record of the row was written by this CTA, into its shared-memory table
       __syncwarp();
-      finalize_row<ES, SAMPLER>(a, row, lane, pre, tb.lrec + (size_t)li * a.nblk * kRecBytes, true, noise);
+      finalize_row<ES, SAMPLER>(a, row, lane, pre, tb.lrec + (size_t)li * a.nblk * kRecBytes, true, true, noise);
       continue;
     }
     const unsigned share = (unsigned)cr.share(k);
+    if (share == (unsigned)a.nblk) {
+      // the row lies wholly inside this CTA's range but did not fit the shared-memory table: its records are in
+      // global memory, all written by this CTA, so no other CTA has to be heard from
+      __syncwarp();
+      finalize_row<ES, SAMPLER>(a, row, lane, pre,
+                                reinterpret_cast<const unsigned char*>(a.records) + (size_t)row * a.nblk * kRecBytes, false,
+                                true, noise);
+      continue;
+    }
     unsigned old = 0;
     if (lane == 0) old = atom_add_acq_rel_gpu(a.ticket + row, share);   // the CTA's records before its ticket
     old = __shfl_sync(kFullMask, old, 0);
@@ -605,7 +614,7 @@ __device__ void drain_queue(const StepArgs& a, const CtaRange& cr, StepCtrl* ctr
     if (old + share == (unsigned)a.nblk)                 // this CTA completed the row
       finalize_row<ES, SAMPLER>(a, row, lane, pre,
                                 reinterpret_cast<const unsigned char*>(a.records) + (size_t)row * a.nblk * kRecBytes, false,
-                                noise);
+                                false, noise);
   }
 }
 
@@ -1111,10 +1120,10 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   const long long qcap = blocks_per_cta / a.nblk + 2;
   if (qcap > kMaxQueue) return ESPO_ERR_CAPACITY;
   a.queue_cap = (int)qcap;
-  // shared-memory table for the records of rows that one CTA reduces alone (at most 16 KB of it)
+  // shared-memory table for the records of rows that one CTA reduces alone (at most 40 KB of it)
   const size_t rec_bytes = (size_t)a.nblk * 16;
   long long local_rows = blocks_per_cta / a.nblk + 1;
-  if ((size_t)local_rows * rec_bytes > 16384) local_rows = (long long)(16384 / rec_bytes);
+  if ((size_t)local_rows * rec_bytes > 40960) local_rows = (long long)(40960 / rec_bytes);
   a.local_rows = (int)local_rows;
   // ... and one for the block-level noise of the rows the range touches (at most 16 KB)
   long long noise_rows = a.queue_cap;
