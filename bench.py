@@ -370,6 +370,36 @@ def main():
                 del sbufs
             out["bandwidth_sweep"] = sweep
 
+            # ---- shrinking active set: as rows stop, the caller passes the n_active surviving rows (compacted
+            #      logits plus the slot list from espo_compact_active); per-step time vs n_active ----
+            act = []
+            sst = espo.espo_init_state(B, V, seed=7)
+            all_ids = torch.arange(B, dtype=torch.int32, device=dev)
+            n_act_dev = torch.zeros(1, dtype=torch.int32, device=dev)
+            for n_act in (B, (3 * B) // 4, B // 2, B // 4, B // 8):
+                ids = all_ids[:n_act].contiguous()
+                for i in range(10):
+                    espo.espo_step(bufs[i % N_BUFFERS][:n_act], values[:n_act], sst, params, tokens, stop, row_ids=ids, n_rows=n_act)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                reps = 200
+                e0.record()
+                for i in range(reps):
+                    espo.espo_step(bufs[i % N_BUFFERS][:n_act], values[:n_act], sst, params, tokens, stop, row_ids=ids, n_rows=n_act)
+                e1.record()
+                torch.cuda.synchronize()
+                us = e0.elapsed_time(e1) * 1e3 / reps
+                act.append({"n_active": n_act, "us": us, "GB/s": n_act * V * 2 / us / 1e3, "rows/s": n_act / (us * 1e-6)})
+            ids_out = torch.empty(B, dtype=torch.int32, device=dev)
+            e0.record()
+            for _ in range(100):
+                espo.espo_compact_active(sst, ids_out, n_act_dev)
+            e1.record()
+            torch.cuda.synchronize()
+            out["active_set"] = {"steps": act, "compact_us": e0.elapsed_time(e1) * 1e3 / 100,
+                                 "note": f"capacity {B} slots, bf16, V={V}; eager launches; compaction is a separate one-CTA kernel"}
+            espo.espo_free_state(sst)
+
         # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region ----
         host_logits = [torch.empty(B, V, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
         for i in range(2):
