@@ -229,15 +229,27 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
     fail_mask &= last_mask;
     double mb = 0.0;
     double vd_next = (double)v_after;
+    if (!__any_sync(kFullMask, last_mask != 0u)) {
+      // no trajectory ends among the warp's 512 tokens (the usual case): no per-token case distinctions
 #pragma unroll
-    for (int e = kAdvPerThread - 1; e >= 0; --e) {
-      const bool last = (last_mask >> e) & 1u;
-      const double vd = (double)v[e];
-      const double rd = ((fail_mask >> e) & 1u) ? r_fail_d : (double)r[e];
-      const double de = (last ? rd : fma(a.gamma, vd_next, rd)) - vd;
-      d[e] = de;
-      mb = last ? de : fma(a.gl, mb, de);
-      vd_next = vd;
+      for (int e = kAdvPerThread - 1; e >= 0; --e) {
+        const double vd = (double)v[e];
+        const double de = fma(a.gamma, vd_next, (double)r[e]) - vd;
+        d[e] = de;
+        mb = fma(a.gl, mb, de);
+        vd_next = vd;
+      }
+    } else {
+#pragma unroll
+      for (int e = kAdvPerThread - 1; e >= 0; --e) {
+        const bool last = (last_mask >> e) & 1u;
+        const double vd = (double)v[e];
+        const double rd = ((fail_mask >> e) & 1u) ? r_fail_d : (double)r[e];
+        const double de = (last ? rd : fma(a.gamma, vd_next, rd)) - vd;
+        d[e] = de;
+        mb = last ? de : fma(a.gl, mb, de);
+        vd_next = vd;
+      }
     }
     // Tokens past the end of the array (only in its last chunk) read as zeros; the array's last token is a
     // forced trajectory end, so nothing of them reaches a stored result.
@@ -312,10 +324,18 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
     // ---- replay the thread's tokens with the value that follows them ----
     double x = fma(after.a, carry_in, after.b);
     float out[kAdvPerThread];
+    if (!__any_sync(kFullMask, last_mask != 0u)) {
 #pragma unroll
-    for (int e = kAdvPerThread - 1; e >= 0; --e) {
-      x = ((last_mask >> e) & 1u) ? d[e] : fma(a.gl, x, d[e]);
-      out[e] = (float)x;
+      for (int e = kAdvPerThread - 1; e >= 0; --e) {
+        x = fma(a.gl, x, d[e]);
+        out[e] = (float)x;
+      }
+    } else {
+#pragma unroll
+      for (int e = kAdvPerThread - 1; e >= 0; --e) {
+        x = ((last_mask >> e) & 1u) ? d[e] : fma(a.gl, x, d[e]);
+        out[e] = (float)x;
+      }
     }
     if (n_in == kAdvPerThread) {
 #pragma unroll
