@@ -39,6 +39,15 @@
 //     g_t = 0, log pi(a_t) = 0.
 //   * a sampled EOS ends the trajectory naturally even if the test would also fire.
 //
+//   * r_fail REPLACES the stored last reward of a stopped trajectory (Eq. 13 sets it).
+//
+// Four of these readings are fixed by nothing the paper prints, and no test can hold them to
+// anything but this file's own statement -- for them parity is "parity unpinned" by the paper:
+// which distribution pi is in Eq. 6 (temperature-scaled here), the values of delta and c in
+// Eq. 9 (run-time parameters), EOS taking precedence over a stop on the same step, and
+// r_fail replacing (not adding to) the stored reward.  Everything else is pinned by the tests
+// (known-answer vectors, library routines, closed forms, invariants, brute force).
+//
 // Everything is brute force over the vocabulary, one row at a time, no blocking or
 // reordering beyond what the definitions above state.
 
