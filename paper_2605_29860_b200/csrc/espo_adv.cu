@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   float* vbuf = rbuf + 2 * kAdvChunk;
   unsigned char* flagbuf = reinterpret_cast<unsigned char*>(vbuf + 2 * kAdvVStride);   // bit0: last token of a trajectory, bit1: it was stopped
   uint64_t* mbar = reinterpret_cast<uint64_t*>(flagbuf + 2 * kAdvChunk);
-  __shared__ Map warp_agg[kAdvWarps];
+  __shared__ Map warp_agg[2][kAdvWarps];                    // double-buffered: consecutive chunks alternate
   __shared__ double pw[kAdvPerThread + 1];                   // (gamma*lambda)^i
   __shared__ double carry_buf[2];                            // value that follows the chunk held by each stage
 
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   // Waits for `stage`, folds the chunk `jj` it holds: leaves the thread's TD errors in d[], its end mask in
   // last_mask, its own map in m and the map of everything after the thread inside the chunk in `after`; the
   // stage's flag bytes are cleared for their next use.  Contains one __syncthreads().
-  auto fold = [&](int jj, int stage) {
+  auto fold = [&](int jj, int stage, int par) {
     const float* rs = rbuf + stage * kAdvChunk;
     const float* vs = vbuf + stage * kAdvVStride;
     const long long p0 = (long long)jj * kAdvChunk;
@@ -260,11 +260,11 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
       Map hi{shfl_down_d(inc.a, o), shfl_down_d(inc.b, o)};
       if (lane + o < 32) inc = compose(inc, hi);
     }
-    if (lane == 0) warp_agg[warp] = inc;
+    if (lane == 0) warp_agg[par][warp] = inc;
     after = Map{shfl_down_d(inc.a, 1), shfl_down_d(inc.b, 1)};   // exclusive within the warp
     if (lane == 31) after = Map{1.0, 0.0};
     __syncthreads();   // warp aggregates written; every thread has read its part of the stage
-    for (int w = warp + 1; w < kAdvWarps; ++w) after = compose(after, warp_agg[w]);
+    for (int w = warp + 1; w < kAdvWarps; ++w) after = compose(after, warp_agg[par][w]);
   };
 
   if (tid == 0) {
@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
       fetch(jh, 0);
       mark_ends(jh, 0);
       __syncthreads();            // flags marked
-      fold(jh, 0);
+      fold(jh, 0, 0);
       const Map whole = compose(m, after);                      // thread 0: the whole chunk
       const double wa = __shfl_sync(kFullMask, whole.a, 0), wb = __shfl_sync(kFullMask, whole.b, 0);
       if (tid == 0) { carry_buf[0] = wa; carry_buf[1] = wb; }
@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
     const int n = (int)min((long long)kAdvChunk, a.total - p0);
     int n_in = n - q0;       // tokens of this thread that exist
     n_in = n_in < 0 ? 0 : (n_in > kAdvPerThread ? kAdvPerThread : n_in);
-    fold(j, s);
+    fold(j, s, s);
     const double carry_in = carry_buf[s];
     if (tid == 0) {
       const Map whole = compose(m, after);
@@ -357,7 +357,8 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
           if (a.ret) a.ret[p0 + q0 + e] = out[e] + __ldcs(a.values + p0 + q0 + e);
         }
     }
-    __syncthreads();   // the next chunk's flags and carry are in place
+    // No barrier here: the next chunk's flags, carry and data are read after the barrier inside its fold(), and
+    // the warp aggregates alternate between two buffers.
   }
 }
 
