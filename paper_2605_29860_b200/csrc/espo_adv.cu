@@ -149,7 +149,9 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
     unsigned char* fl = flagbuf + stage * kAdvChunk;
     const long long p0 = (long long)jj * kAdvChunk;
     const long long p_end = min(p0 + kAdvChunk, a.total);
-    for (int i = __ldg(a.ws.chunk_first + jj) + tid; i < a.B; i += kAdvThreads) {
+    int first = __ldcg(a.ws.chunk_first + jj);
+    if ((unsigned)first >= (unsigned)a.B) first = a.B;   // only with inconsistent lengths (flagged by the preparation)
+    for (int i = first + tid; i < a.B; i += kAdvThreads) {
       const long long o0 = __ldcg(a.ws.offsets + i);
       const long long o1 = __ldcg(a.ws.offsets + i + 1);
       const unsigned st = a.stopped[i];
@@ -279,33 +281,75 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   __syncthreads();
   if (c_lo >= c_hi) return;
 
-  // ---- the value that follows the CTA's highest chunk: fold the rest of the trajectory that crosses the range's
-  //      upper end (chunks c_hi, c_hi + 1, ... up to the first one that holds a trajectory end).  Stage 1 meanwhile
-  //      receives the highest chunk of the range. ----
+  // ---- the two highest chunks of the range are on their way while the CTA works out what follows the range ----
   fetch(c_hi - 1, 1);
+  if (c_hi - 2 >= c_lo) fetch(c_hi - 2, 0);
   mark_ends(c_hi - 1, 1);
-  double carry = 0.0;
+  if (c_hi - 2 >= c_lo) mark_ends(c_hi - 2, 0);
+
+  // ---- the advantage of the token that follows the range (token c_hi * kAdvChunk).  Its trajectory continues in the
+  //      next CTA's range; unrolled, Eq. 5 makes it the weighted sum of the rest of that one trajectory's TD errors,
+  //      sum_k (gamma*lambda)^k delta_k, which the CTA's threads take straight from global memory (read only, usually
+  //      served by L2): thread t owns tokens 4t .. 4t+3 of every 1024.  CTAs therefore never wait for one another. ----
   {
-    Map acc{1.0, 0.0};
-    for (int jh = c_hi; jh < a.nchunks && acc.a != 0.0; ++jh) {
-      fetch(jh, 0);
-      mark_ends(jh, 0);
-      __syncthreads();            // flags marked
-      fold(jh, 0, 0);
-      const Map whole = compose(m, after);                      // thread 0: the whole chunk
-      const double wa = __shfl_sync(kFullMask, whole.a, 0), wb = __shfl_sync(kFullMask, whole.b, 0);
-      if (tid == 0) { carry_buf[0] = wa; carry_buf[1] = wb; }
-      __syncthreads();
-      acc = compose(acc, Map{carry_buf[0], carry_buf[1]});
-      __syncthreads();            // carry_buf free again
+    double part = 0.0;
+    const long long P = (long long)c_hi * kAdvChunk;
+    if (c_hi < a.nchunks) {
+      const int i = __ldcg(a.ws.chunk_first + c_hi);
+      if ((unsigned)i < (unsigned)a.B) {
+        const long long end = min(__ldcg(a.ws.offsets + i + 1), a.total);
+        const bool failed = a.stopped[i] != 0;
+        double wt = 1.0, sq = a.gl;                        // (gamma*lambda)^(4 tid) by binary powering
+        for (unsigned ex = 4u * tid; ex; ex >>= 1) {
+          if (ex & 1u) wt *= sq;
+          sq *= sq;
+        }
+        double w_round = a.gl;                             // (gamma*lambda)^(4 * kAdvThreads)
+#pragma unroll
+        for (int h = 0; h < 10; ++h) w_round *= w_round;
+        static_assert(4 * kAdvThreads == 1024, "w_round is the 1024th power");
+#pragma unroll 2
+        for (long long k0 = P + 4 * tid; k0 < end; k0 += 4 * kAdvThreads, wt *= w_round) {
+          float r[4], v[5];
+          if (k0 + 4 < a.total) {                          // four tokens and the value after them exist
+            const float4 rr = __ldg(reinterpret_cast<const float4*>(a.rewards + k0));
+            const float4 vv = __ldg(reinterpret_cast<const float4*>(a.values + k0));
+            v[4] = __ldg(a.values + k0 + 4);
+            r[0] = rr.x; r[1] = rr.y; r[2] = rr.z; r[3] = rr.w;
+            v[0] = vv.x; v[1] = vv.y; v[2] = vv.z; v[3] = vv.w;
+          } else {
+#pragma unroll
+            for (int e = 0; e < 5; ++e) {
+              v[e] = (k0 + e < a.total) ? __ldg(a.values + k0 + e) : 0.f;
+              if (e < 4) r[e] = (k0 + e < a.total) ? __ldg(a.rewards + k0 + e) : 0.f;
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const long long k = k0 + e;
+            if (k < end) {
+              const bool last = (k == end - 1);
+              const double rd = (last && failed) ? r_fail_d : (double)r[e];
+              const double de = (last ? rd : fma(a.gamma, (double)v[e + 1], rd)) - (double)v[e];
+              part = fma(wt * pw[e], de, part);
+            }
+          }
+        }
+      }
     }
-    carry = acc.b;                // past the end of the array the value is 0
+#pragma unroll
+    for (int o = 16; o; o >>= 1) part += shfl_down_d(part, o);
+    if (lane == 0) warp_agg[0][warp].b = part;
+    __syncthreads();
+    if (tid == 0) {
+      double carry = 0.0;                                  // past the end of the array the value is 0
+      for (int w = 0; w < kAdvWarps; ++w) carry += warp_agg[0][w].b;
+      carry_buf[1] = carry;
+    }
   }
-  if (tid == 0) carry_buf[1] = carry;
+  __syncthreads();   // carry, flags of both stages
 
   // ---- the range, from its highest chunk down; chunk j sits in stage (c_hi - 1 - j + 1) & 1 ----
-  if (c_hi - 2 >= c_lo) { fetch(c_hi - 2, 0); mark_ends(c_hi - 2, 0); }
-  __syncthreads();
   int s = 1;
   for (int j = c_hi - 1; j >= c_lo; --j, s ^= 1) {
     const long long p0 = (long long)j * kAdvChunk;
