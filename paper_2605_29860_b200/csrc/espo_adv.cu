@@ -19,6 +19,7 @@
 // A small preparation kernel turns lengths into offsets and tells every chunk which
 // trajectory its first token belongs to.
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdint.h>
 #include <string.h>
 
@@ -55,6 +56,7 @@ struct AdvArgs {
   long long total;
   int nchunks;
   double gamma, gl;       // gamma, gamma*lambda
+  long long halo_cap;     // tokens of a crossing trajectory whose weight (gamma*lambda)^k can still matter
   float r_fail;
   AdvWorkspace ws;
 };
@@ -67,6 +69,9 @@ __global__ void __launch_bounds__(kPrepThreads) espo_adv_prep_kernel(const AdvAr
   __shared__ long long warp_tot[32];
   __shared__ long long carry;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // The scan kernel may be scheduled now: it starts its first copies and waits for this grid before it reads
+  // anything written here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) carry = 0;
   __syncthreads();
   bool bad = false;
@@ -110,6 +115,20 @@ __global__ void __launch_bounds__(kPrepThreads) espo_adv_prep_kernel(const AdvAr
 // The scan.
 // ---------------------------------------------------------------------------------------
 
+// Fills the discount fields.  (gamma*lambda)^k < 2^-80 from k = halo_cap on: such a term cannot move a sum of TD
+// errors by more than 2^-80 times the largest of them, far below the rounding of the double-precision sum itself.
+static void set_discount(AdvArgs& a, float gamma, float lambda) {
+  a.gamma = (double)gamma;
+  a.gl = (double)gamma * (double)lambda;
+  const double g = a.gl < 0 ? -a.gl : a.gl;
+  if (g >= 1.0) a.halo_cap = 0x7fffffffffffffffLL;
+  else if (g <= 0.0) a.halo_cap = 1;
+  else {
+    const double k = -80.0 * 0.6931471805599453 / log(g);
+    a.halo_cap = k < 1e15 ? (long long)k + 1 : 0x7fffffffffffffffLL;
+  }
+}
+
 struct Map {   // X -> b + a * X
   double a, b;
 };
@@ -134,54 +153,65 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   __shared__ Map warp_agg[2][kAdvWarps];                    // double-buffered: consecutive chunks alternate
   __shared__ double pw[kAdvPerThread + 1];                   // (gamma*lambda)^i
   __shared__ double carry_buf[2];                            // value that follows the chunk held by each stage
+  __shared__ int halo_traj;                                  // trajectory that crosses the range's upper end, or -1
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const double r_fail_d = (double)a.r_fail;
   const int q0 = tid * kAdvPerThread;
 
-  // this CTA's chunks: [c_lo, c_hi), walked from c_hi - 1 down
-  const int c_lo = (int)((long long)blockIdx.x * a.nchunks / gridDim.x);
-  const int c_hi = (int)((long long)(blockIdx.x + 1) * a.nchunks / gridDim.x);
+  // This CTA's tokens: [t_lo, t_hi), cut at multiples of four tokens so that every CTA moves the same number of
+  // bytes and every copy starts on a 16-byte boundary (the last range ends at the array's end rounded up).  Chunk k
+  // (k = 0 is the highest) covers tokens [t_hi - (k+1)*kAdvChunk, t_hi - k*kAdvChunk); the lowest chunk may begin
+  // below t_lo: those positions of its stage are never loaded, and what the threads compute for them is dropped.
+  const long long quads = (a.total + 3) >> 2;
+  const long long t_lo = 4 * ((long long)blockIdx.x * quads / gridDim.x);
+  const long long t_hi = 4 * ((long long)(blockIdx.x + 1) * quads / gridDim.x);
+  const int nck = (int)((t_hi - t_lo + kAdvChunk - 1) / kAdvChunk);
 
-  // Marks the trajectory ends that fall into chunk `jj` in the flag bytes of `stage`.  The three loads of a
+  // Marks the trajectory ends that fall into chunk `k` in the flag bytes of `stage`.  The three loads of a
   // trajectory are independent of one another.
-  auto mark_ends = [&](int jj, int stage) {
+  auto mark_ends = [&](int k, int stage) {
     unsigned char* fl = flagbuf + stage * kAdvChunk;
-    const long long p0 = (long long)jj * kAdvChunk;
+    const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+    const long long p_lo = max(p0, t_lo);
     const long long p_end = min(p0 + kAdvChunk, a.total);
-    int first = __ldcg(a.ws.chunk_first + jj);
-    if ((unsigned)first >= (unsigned)a.B) first = a.B;   // only with inconsistent lengths (flagged by the preparation)
+    int first = __ldcg(a.ws.chunk_first + (p_lo / kAdvChunk));   // the trajectory of a token at or below p_lo
+    if ((unsigned)first >= (unsigned)a.B) first = a.B;           // only with inconsistent lengths (flagged by the preparation)
     for (int i = first + tid; i < a.B; i += kAdvThreads) {
       const long long o0 = __ldcg(a.ws.offsets + i);
       const long long o1 = __ldcg(a.ws.offsets + i + 1);
       const unsigned st = a.stopped[i];
       if (o0 >= p_end) break;
-      if (o1 > o0 && o1 - 1 >= p0 && o1 - 1 < p_end) fl[o1 - 1 - p0] = (unsigned char)(1u | (st ? 2u : 0u));
+      if (o1 > o0 && o1 - 1 >= p_lo && o1 - 1 < p_end) fl[o1 - 1 - p0] = (unsigned char)(1u | (st ? 2u : 0u));
     }
   };
 
-  // Starts the copy of chunk `jj` into `stage`; called by every thread.  A full chunk is two bulk copies
-  // (plus 16 bytes for the value after the chunk) that complete on the stage's mbarrier; the array's ragged
-  // last chunk is copied with ordinary loads and the barrier completed by hand.
-  auto fetch = [&](int jj, int stage) {
-    const long long p0 = (long long)jj * kAdvChunk;
+  // Starts the copy of chunk `k` into `stage`; called by every thread.  A chunk is two bulk copies (plus 16 bytes
+  // for the value after the chunk) that complete on the stage's mbarrier; a chunk that reaches past the end of the
+  // array (only the array's last, when its length is no multiple of four) is copied with ordinary loads and the
+  // barrier completed by hand.
+  auto fetch = [&](int k, int stage) {
+    const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+    const int skip = (int)(max(p0, t_lo) - p0);                    // unused positions at the low end, a multiple of 4
     float* rs = rbuf + stage * kAdvChunk;
     float* vs = vbuf + stage * kAdvVStride;
     if (p0 + kAdvChunk <= a.total) {
       if (tid == 0) {
         const bool tail16 = (p0 + kAdvChunk + 4 <= a.total);      // the 16 bytes after the chunk exist
+        const uint32_t bytes = (uint32_t)sizeof(float) * (uint32_t)(kAdvChunk - skip);
         fence_proxy_async();                                       // earlier reads of the stage come first
-        mbar_arrive_expect_tx(&mbar[stage], 2u * sizeof(float) * kAdvChunk + (tail16 ? 16u : 0u));
-        bulk_copy_g2s(rs, a.rewards + p0, sizeof(float) * kAdvChunk, &mbar[stage]);
-        bulk_copy_g2s(vs, a.values + p0, sizeof(float) * kAdvChunk, &mbar[stage]);
+        mbar_arrive_expect_tx(&mbar[stage], 2u * bytes + (tail16 ? 16u : 0u));
+        bulk_copy_g2s(rs + skip, a.rewards + p0 + skip, bytes, &mbar[stage]);
+        bulk_copy_g2s(vs + skip, a.values + p0 + skip, bytes, &mbar[stage]);
         if (tail16) bulk_copy_g2s(vs + kAdvChunk, a.values + p0 + kAdvChunk, 16u, &mbar[stage]);
         else vs[kAdvChunk] = (p0 + kAdvChunk < a.total) ? __ldg(a.values + p0 + kAdvChunk) : 0.f;
       }
     } else {
       const int n = (int)(a.total - p0);
       for (int q = tid; q < kAdvChunk; q += kAdvThreads) {
-        rs[q] = (q < n) ? __ldcs(a.rewards + p0 + q) : 0.f;
-        vs[q] = (q < n) ? __ldcs(a.values + p0 + q) : 0.f;
+        const bool ok = q >= skip && q < n;
+        rs[q] = ok ? __ldcs(a.rewards + p0 + q) : 0.f;
+        vs[q] = ok ? __ldcs(a.values + p0 + q) : 0.f;
       }
       if (tid == 0) vs[kAdvChunk] = 0.f;
       __syncthreads();
@@ -194,13 +224,13 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   double d[kAdvPerThread];
   Map m, after;
 
-  // Waits for `stage`, folds the chunk `jj` it holds: leaves the thread's TD errors in d[], its end mask in
+  // Waits for `stage`, folds the chunk `k` it holds: leaves the thread's TD errors in d[], its end mask in
   // last_mask, its own map in m and the map of everything after the thread inside the chunk in `after`; the
   // stage's flag bytes are cleared for their next use.  Contains one __syncthreads().
-  auto fold = [&](int jj, int stage, int par) {
+  auto fold = [&](int k, int stage, int par) {
     const float* rs = rbuf + stage * kAdvChunk;
     const float* vs = vbuf + stage * kAdvVStride;
-    const long long p0 = (long long)jj * kAdvChunk;
+    const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
     if (!mbar_wait_bounded(&mbar[stage], phase[stage], nullptr)) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
     phase[stage] ^= 1u;
     float r[kAdvPerThread], v[kAdvPerThread];
@@ -270,6 +300,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   };
 
   if (tid == 0) {
+    halo_traj = -1;
     mbar_init(&mbar[0], 1);
     mbar_init(&mbar[1], 1);
     mbar_init_fence();
@@ -279,60 +310,72 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   reinterpret_cast<uint4*>(flagbuf)[tid] = make_uint4(0u, 0u, 0u, 0u);
   reinterpret_cast<uint4*>(flagbuf)[tid + kAdvThreads] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
-  if (c_lo >= c_hi) return;
+  if (nck <= 0) return;
 
   // ---- the two highest chunks of the range are on their way while the CTA works out what follows the range ----
-  fetch(c_hi - 1, 1);
-  if (c_hi - 2 >= c_lo) fetch(c_hi - 2, 0);
-  mark_ends(c_hi - 1, 1);
-  if (c_hi - 2 >= c_lo) mark_ends(c_hi - 2, 0);
+  fetch(0, 1);
+  if (nck > 1) fetch(1, 0);
+  // Launched as a programmatic dependent of the preparation kernel: everything above overlaps with it, everything
+  // below reads what it wrote.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  mark_ends(0, 1);
+  if (nck > 1) mark_ends(1, 0);
 
-  // ---- the advantage of the token that follows the range (token c_hi * kAdvChunk).  Its trajectory continues in the
-  //      next CTA's range; unrolled, Eq. 5 makes it the weighted sum of the rest of that one trajectory's TD errors,
+  // ---- the advantage of the token that follows the range (token t_hi).  Its trajectory continues in the next CTA's
+  //      range; unrolled, Eq. 5 makes it the weighted sum of the rest of that one trajectory's TD errors,
   //      sum_k (gamma*lambda)^k delta_k, which the CTA's threads take straight from global memory (read only, usually
   //      served by L2): thread t owns tokens 4t .. 4t+3 of every 1024.  CTAs therefore never wait for one another. ----
+  if (t_hi < a.total) {   // find the trajectory that holds token t_hi
+    int first = __ldcg(a.ws.chunk_first + (t_hi / kAdvChunk));
+    if ((unsigned)first >= (unsigned)a.B) first = a.B;
+    for (int i = first + tid; i < a.B; i += kAdvThreads) {
+      const long long o0 = __ldcg(a.ws.offsets + i);
+      const long long o1 = __ldcg(a.ws.offsets + i + 1);
+      if (o0 > t_hi) break;
+      if (o1 > t_hi) halo_traj = i;
+    }
+  }
+  __syncthreads();
   {
     double part = 0.0;
-    const long long P = (long long)c_hi * kAdvChunk;
-    if (c_hi < a.nchunks) {
-      const int i = __ldcg(a.ws.chunk_first + c_hi);
-      if ((unsigned)i < (unsigned)a.B) {
-        const long long end = min(__ldcg(a.ws.offsets + i + 1), a.total);
-        const bool failed = a.stopped[i] != 0;
-        double wt = 1.0, sq = a.gl;                        // (gamma*lambda)^(4 tid) by binary powering
-        for (unsigned ex = 4u * tid; ex; ex >>= 1) {
-          if (ex & 1u) wt *= sq;
-          sq *= sq;
-        }
-        double w_round = a.gl;                             // (gamma*lambda)^(4 * kAdvThreads)
+    const int i = halo_traj;
+    if (i >= 0) {
+      const long long t_end = min(__ldcg(a.ws.offsets + i + 1), a.total);          // the trajectory's end
+      const long long end = (t_end - t_hi > a.halo_cap) ? t_hi + a.halo_cap : t_end; // the part whose weights matter
+      const bool failed = a.stopped[i] != 0;
+      double wt = 1.0, sq = a.gl;                        // (gamma*lambda)^(4 tid) by binary powering
+      for (unsigned ex = 4u * tid; ex; ex >>= 1) {
+        if (ex & 1u) wt *= sq;
+        sq *= sq;
+      }
+      double w_round = a.gl;                             // (gamma*lambda)^(4 * kAdvThreads)
 #pragma unroll
-        for (int h = 0; h < 10; ++h) w_round *= w_round;
-        static_assert(4 * kAdvThreads == 1024, "w_round is the 1024th power");
-#pragma unroll 2
-        for (long long k0 = P + 4 * tid; k0 < end; k0 += 4 * kAdvThreads, wt *= w_round) {
-          float r[4], v[5];
-          if (k0 + 4 < a.total) {                          // four tokens and the value after them exist
-            const float4 rr = __ldg(reinterpret_cast<const float4*>(a.rewards + k0));
-            const float4 vv = __ldg(reinterpret_cast<const float4*>(a.values + k0));
-            v[4] = __ldg(a.values + k0 + 4);
-            r[0] = rr.x; r[1] = rr.y; r[2] = rr.z; r[3] = rr.w;
-            v[0] = vv.x; v[1] = vv.y; v[2] = vv.z; v[3] = vv.w;
-          } else {
+      for (int h = 0; h < 10; ++h) w_round *= w_round;
+      static_assert(4 * kAdvThreads == 1024, "w_round is the 1024th power");
+#pragma unroll 4
+      for (long long k0 = t_hi + 4 * tid; k0 < end; k0 += 4 * kAdvThreads, wt *= w_round) {
+        float r[4], v[5];
+        if (k0 + 4 < a.total) {                          // four tokens and the value after them exist
+          const float4 rr = __ldg(reinterpret_cast<const float4*>(a.rewards + k0));
+          const float4 vv = __ldg(reinterpret_cast<const float4*>(a.values + k0));
+          v[4] = __ldg(a.values + k0 + 4);
+          r[0] = rr.x; r[1] = rr.y; r[2] = rr.z; r[3] = rr.w;
+          v[0] = vv.x; v[1] = vv.y; v[2] = vv.z; v[3] = vv.w;
+        } else {
 #pragma unroll
-            for (int e = 0; e < 5; ++e) {
-              v[e] = (k0 + e < a.total) ? __ldg(a.values + k0 + e) : 0.f;
-              if (e < 4) r[e] = (k0 + e < a.total) ? __ldg(a.rewards + k0 + e) : 0.f;
-            }
+          for (int e = 0; e < 5; ++e) {
+            v[e] = (k0 + e < a.total) ? __ldg(a.values + k0 + e) : 0.f;
+            if (e < 4) r[e] = (k0 + e < a.total) ? __ldg(a.rewards + k0 + e) : 0.f;
           }
+        }
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const long long k = k0 + e;
-            if (k < end) {
-              const bool last = (k == end - 1);
-              const double rd = (last && failed) ? r_fail_d : (double)r[e];
-              const double de = (last ? rd : fma(a.gamma, (double)v[e + 1], rd)) - (double)v[e];
-              part = fma(wt * pw[e], de, part);
-            }
+        for (int e = 0; e < 4; ++e) {
+          const long long k = k0 + e;
+          if (k < end) {
+            const bool last = (k == t_end - 1);
+            const double rd = (last && failed) ? r_fail_d : (double)r[e];
+            const double de = (last ? rd : fma(a.gamma, (double)v[e + 1], rd)) - (double)v[e];
+            part = fma(wt * pw[e], de, part);
           }
         }
       }
@@ -349,21 +392,20 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   }
   __syncthreads();   // carry, flags of both stages
 
-  // ---- the range, from its highest chunk down; chunk j sits in stage (c_hi - 1 - j + 1) & 1 ----
+  // ---- the range, from its highest chunk down; chunk k sits in stage (k + 1) & 1 ----
   int s = 1;
-  for (int j = c_hi - 1; j >= c_lo; --j, s ^= 1) {
-    const long long p0 = (long long)j * kAdvChunk;
-    const int n = (int)min((long long)kAdvChunk, a.total - p0);
-    int n_in = n - q0;       // tokens of this thread that exist
-    n_in = n_in < 0 ? 0 : (n_in > kAdvPerThread ? kAdvPerThread : n_in);
-    fold(j, s, s);
+  for (int k = 0; k < nck; ++k, s ^= 1) {
+    const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+    const int q_lo = (int)(max(p0, t_lo) - p0);                               // positions [q_lo, q_hi) hold this
+    const int q_hi = (int)min((long long)kAdvChunk, a.total - p0);           // CTA's tokens
+    fold(k, s, s);
     const double carry_in = carry_buf[s];
     if (tid == 0) {
       const Map whole = compose(m, after);
       carry_buf[s ^ 1] = fma(whole.a, carry_in, whole.b);       // what follows the next (lower) chunk
     }
     // the stage is free: start the copy of the chunk two below, and mark its trajectory ends
-    if (j - 2 >= c_lo) { fetch(j - 2, s); mark_ends(j - 2, s); }
+    if (k + 2 < nck) { fetch(k + 2, s); mark_ends(k + 2, s); }
 
     // ---- replay the thread's tokens with the value that follows them ----
     double x = fma(after.a, carry_in, after.b);
@@ -381,7 +423,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
         out[e] = (float)x;
       }
     }
-    if (n_in == kAdvPerThread) {
+    if (q0 >= q_lo && q0 + kAdvPerThread <= q_hi) {
 #pragma unroll
       for (int h = 0; h < kAdvPerThread / 4; ++h)
         __stcs(reinterpret_cast<float4*>(a.adv + p0 + q0) + h, make_float4(out[4 * h], out[4 * h + 1], out[4 * h + 2], out[4 * h + 3]));
@@ -396,7 +438,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
     } else {
 #pragma unroll
       for (int e = 0; e < kAdvPerThread; ++e)
-        if (e < n_in) {
+        if (q0 + e >= q_lo && q0 + e < q_hi) {
           a.adv[p0 + q0 + e] = out[e];
           if (a.ret) a.ret[p0 + q0 + e] = out[e] + __ldcs(a.values + p0 + q0 + e);
         }
@@ -420,8 +462,17 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
   ESPO_CUDA_TRY(cudaGetLastError());
   long long grid = (long long)sm_count * kAdvCtasPerSm;
   if (grid > a.nchunks) grid = a.nchunks;
-  espo_adv_scan_kernel<<<(unsigned)grid, kAdvThreads, kAdvSmemBytes, s>>>(a);
-  ESPO_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kAdvThreads);
+  cfg.dynamicSmemBytes = kAdvSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start before the preparation kernel ends
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel, a));
   return ESPO_OK;
 }
 
@@ -522,7 +573,7 @@ int espo_advantages_noalloc(const float* rewards, const float* values, const int
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = nullptr;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
-  a.gamma = (double)gamma; a.gl = (double)gamma * (double)lambda;
+  set_discount(a, gamma, lambda);
   a.r_fail = r_fail;
   a.ws.offsets = (long long*)(b + kNaOffOffsets);
   a.ws.chunk_first = (int*)(b + kNaOffChunkFirst);
@@ -563,7 +614,7 @@ int espo_advantages_returns(const float* rewards, const float* values, const int
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = returns_out;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
-  a.gamma = (double)gamma; a.gl = (double)gamma * (double)lambda;
+  set_discount(a, gamma, lambda);
   a.r_fail = r_fail;
   a.ws = p->ws;
   return launch_advantages(a, p->sm_count, s);
