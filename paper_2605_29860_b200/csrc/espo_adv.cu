@@ -31,11 +31,13 @@
 
 namespace espo {
 
-constexpr int kAdvThreads = 256;
+constexpr int kAdvThreads = 256;                        // scanning threads
 constexpr int kAdvPerThread = 16;
 constexpr int kAdvChunk = kAdvThreads * kAdvPerThread;   // 4096 tokens
 constexpr int kAdvWarps = kAdvThreads / 32;
-constexpr int kAdvCtasPerSm = 3;
+constexpr int kAdvCtaThreads = kAdvThreads + 32;          // the scanning threads and the producer warp
+constexpr int kAdvStages = 3;
+constexpr int kAdvCtasPerSm = 2;
 constexpr int kMaxDevicesAdv = 64;
 constexpr int kPrepThreads = 1024;
 
@@ -139,21 +141,29 @@ __device__ __forceinline__ double shfl_down_d(double v, int o) { return __shfl_d
 __device__ __forceinline__ double shfl_up_d(double v, int o) { return __shfl_up_sync(kFullMask, v, o); }
 __device__ __forceinline__ double shfl_d(double v, int src) { return __shfl_sync(kFullMask, v, src); }
 
-// Shared memory of the scan kernel: two stages, each one chunk of rewards, one chunk of values followed by the
-// value of the token after the chunk, and one flag byte per token.
-constexpr int kAdvVStride = kAdvChunk + 4;      // floats; keeps the second stage 16-byte aligned
-constexpr size_t kAdvSmemBytes = 2 * sizeof(float) * kAdvChunk + 2 * sizeof(float) * kAdvVStride + 2 * kAdvChunk + 2 * sizeof(uint64_t);
+// Shared memory of the scan kernel: a ring of kAdvStages stages, each one chunk of rewards, one chunk of values
+// followed by the value of the token after the chunk, and one flag word per scanning thread (bit e: the thread's
+// token e is the last of a trajectory; bit 16 + e: that trajectory was stopped).
+constexpr int kAdvVStride = kAdvChunk + 4;      // floats; keeps every stage 16-byte aligned
+constexpr size_t kAdvSmemBytes =
+    (size_t)kAdvStages * (sizeof(float) * kAdvChunk + sizeof(float) * kAdvVStride + sizeof(uint32_t) * kAdvThreads) +
+    2 * kAdvStages * sizeof(uint64_t);
 
-__global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kernel(const AdvArgs a) {
+// kAdvThreads threads scan; one more warp (the producer) keeps the ring full and sets the flag words, so that no
+// scanning warp ever waits for a load from global memory.
+__global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_kernel(const AdvArgs a) {
   extern __shared__ __align__(128) unsigned char adv_smem[];
   float* rbuf = reinterpret_cast<float*>(adv_smem);
-  float* vbuf = rbuf + 2 * kAdvChunk;
-  unsigned char* flagbuf = reinterpret_cast<unsigned char*>(vbuf + 2 * kAdvVStride);   // bit0: last token of a trajectory, bit1: it was stopped
-  uint64_t* mbar = reinterpret_cast<uint64_t*>(flagbuf + 2 * kAdvChunk);
+  float* vbuf = rbuf + kAdvStages * kAdvChunk;
+  uint32_t* fwbuf = reinterpret_cast<uint32_t*>(vbuf + kAdvStages * kAdvVStride);
+  uint64_t* full = reinterpret_cast<uint64_t*>(fwbuf + kAdvStages * kAdvThreads);   // data and flags of the stage are in place
+  uint64_t* empty = full + kAdvStages;                                                // every scanning thread has read the stage
   __shared__ Map warp_agg[2][kAdvWarps];                    // double-buffered: consecutive chunks alternate
   __shared__ double pw[kAdvPerThread + 1];                   // (gamma*lambda)^i
-  __shared__ double carry_buf[2];                            // value that follows the chunk held by each stage
-  __shared__ int halo_traj;                                  // trajectory that crosses the range's upper end, or -1
+  __shared__ double carry_buf[2];                            // value that follows the chunk, by the chunk's parity
+  __shared__ int halo_traj;                                  // trajectory that crosses the range's upper end, or -1,
+  __shared__ long long halo_end;                             // its end offset
+  __shared__ int halo_failed;                                // and whether it was stopped
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const double r_fail_d = (double)a.r_fail;
@@ -161,78 +171,133 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
 
   // This CTA's tokens: [t_lo, t_hi), cut at multiples of four tokens so that every CTA moves the same number of
   // bytes and every copy starts on a 16-byte boundary (the last range ends at the array's end rounded up).  Chunk k
-  // (k = 0 is the highest) covers tokens [t_hi - (k+1)*kAdvChunk, t_hi - k*kAdvChunk); the lowest chunk may begin
-  // below t_lo: those positions of its stage are never loaded, and what the threads compute for them is dropped.
+  // (k = 0 is the highest) covers tokens [t_hi - (k+1)*kAdvChunk, t_hi - k*kAdvChunk) and sits in stage k mod
+  // kAdvStages; the lowest chunk may begin below t_lo: those positions of its stage are never loaded, and what the
+  // threads compute for them is dropped.
   const long long quads = (a.total + 3) >> 2;
   const long long t_lo = 4 * ((long long)blockIdx.x * quads / gridDim.x);
   const long long t_hi = 4 * ((long long)(blockIdx.x + 1) * quads / gridDim.x);
   const int nck = (int)((t_hi - t_lo + kAdvChunk - 1) / kAdvChunk);
 
-  // Marks the trajectory ends that fall into chunk `k` in the flag bytes of `stage`.  The three loads of a
-  // trajectory are independent of one another.
-  auto mark_ends = [&](int k, int stage) {
-    unsigned char* fl = flagbuf + stage * kAdvChunk;
-    const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
-    const long long p_lo = max(p0, t_lo);
-    const long long p_end = min(p0 + kAdvChunk, a.total);
-    int first = __ldcg(a.ws.chunk_first + (p_lo / kAdvChunk));   // the trajectory of a token at or below p_lo
-    if ((unsigned)first >= (unsigned)a.B) first = a.B;           // only with inconsistent lengths (flagged by the preparation)
-    for (int i = first + tid; i < a.B; i += kAdvThreads) {
-      const long long o0 = __ldcg(a.ws.offsets + i);
-      const long long o1 = __ldcg(a.ws.offsets + i + 1);
-      const unsigned st = a.stopped[i];
-      if (o0 >= p_end) break;
-      if (o1 > o0 && o1 - 1 >= p_lo && o1 - 1 < p_end) fl[o1 - 1 - p0] = (unsigned char)(1u | (st ? 2u : 0u));
+  if (tid == 0) {
+    halo_traj = -1;
+    for (int st = 0; st < kAdvStages; ++st) {
+      mbar_init(&full[st], 2);               // the producer's expect_tx arrival and its arrival after the flags
+      mbar_init(&empty[st], kAdvThreads);
     }
-  };
+    mbar_init_fence();
+    double p = 1.0;
+    for (int i = 0; i <= kAdvPerThread; ++i) { pw[i] = p; p *= a.gl; }
+  }
+  for (int i = tid; i < kAdvStages * kAdvThreads; i += kAdvCtaThreads) fwbuf[i] = 0u;
+  __syncthreads();
+  if (nck <= 0) return;
 
-  // Starts the copy of chunk `k` into `stage`; called by every thread.  A chunk is two bulk copies (plus 16 bytes
-  // for the value after the chunk) that complete on the stage's mbarrier; a chunk that reaches past the end of the
-  // array (only the array's last, when its length is no multiple of four) is copied with ordinary loads and the
-  // barrier completed by hand.
-  auto fetch = [&](int k, int stage) {
-    const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
-    const int skip = (int)(max(p0, t_lo) - p0);                    // unused positions at the low end, a multiple of 4
-    float* rs = rbuf + stage * kAdvChunk;
-    float* vs = vbuf + stage * kAdvVStride;
-    if (p0 + kAdvChunk <= a.total) {
-      if (tid == 0) {
-        const bool tail16 = (p0 + kAdvChunk + 4 <= a.total);      // the 16 bytes after the chunk exist
-        const uint32_t bytes = (uint32_t)sizeof(float) * (uint32_t)(kAdvChunk - skip);
-        fence_proxy_async();                                       // earlier reads of the stage come first
-        mbar_arrive_expect_tx(&mbar[stage], 2u * bytes + (tail16 ? 16u : 0u));
-        bulk_copy_g2s(rs + skip, a.rewards + p0 + skip, bytes, &mbar[stage]);
-        bulk_copy_g2s(vs + skip, a.values + p0 + skip, bytes, &mbar[stage]);
-        if (tail16) bulk_copy_g2s(vs + kAdvChunk, a.values + p0 + kAdvChunk, 16u, &mbar[stage]);
-        else vs[kAdvChunk] = (p0 + kAdvChunk < a.total) ? __ldg(a.values + p0 + kAdvChunk) : 0.f;
+  if (warp == kAdvWarps) {
+    // =============================== producer warp ===============================
+    // Starts the copies of chunk `k` (lane 0).  A chunk is two bulk copies (plus 16 bytes for the value after the
+    // chunk) that complete on the stage's mbarrier; of a chunk that reaches past the end of the array (only the
+    // array's last, when its length is no multiple of four) the last, incomplete group of four tokens is written
+    // with ordinary stores, zeros standing for the tokens that do not exist.
+    auto issue_copies = [&](int k) {
+      const int stage = k % kAdvStages;
+      const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+      const int skip = (int)(max(p0, t_lo) - p0);                        // unused positions at the low end, a multiple of 4
+      const int n = (int)min((long long)kAdvChunk, a.total - p0);       // positions below n hold tokens
+      const int n4 = n & ~3;
+      float* rs = rbuf + stage * kAdvChunk;
+      float* vs = vbuf + stage * kAdvVStride;
+      const bool tail16 = (p0 + kAdvChunk + 4 <= a.total);               // the 16 bytes after the chunk exist
+      const uint32_t bytes = n4 > skip ? (uint32_t)sizeof(float) * (uint32_t)(n4 - skip) : 0u;
+      fence_proxy_async();                                               // the scanning threads' reads of the stage come first
+      mbar_arrive_expect_tx(&full[stage], 2u * bytes + (tail16 ? 16u : 0u));
+      if (bytes) {
+        bulk_copy_g2s(rs + skip, a.rewards + p0 + skip, bytes, &full[stage]);
+        bulk_copy_g2s(vs + skip, a.values + p0 + skip, bytes, &full[stage]);
       }
-    } else {
-      const int n = (int)(a.total - p0);
-      for (int q = tid; q < kAdvChunk; q += kAdvThreads) {
-        const bool ok = q >= skip && q < n;
-        rs[q] = ok ? __ldcs(a.rewards + p0 + q) : 0.f;
-        vs[q] = ok ? __ldcs(a.values + p0 + q) : 0.f;
+      if (tail16) bulk_copy_g2s(vs + kAdvChunk, a.values + p0 + kAdvChunk, 16u, &full[stage]);
+      else vs[kAdvChunk] = (p0 + kAdvChunk < a.total) ? __ldg(a.values + p0 + kAdvChunk) : 0.f;
+      for (int q = n4; q < n4 + 4 && q < kAdvChunk; ++q) {
+        rs[q] = (q < n) ? __ldg(a.rewards + p0 + q) : 0.f;
+        vs[q] = (q < n) ? __ldg(a.values + p0 + q) : 0.f;
       }
-      if (tid == 0) vs[kAdvChunk] = 0.f;
-      __syncthreads();
-      if (tid == 0) mbar_arrive(&mbar[stage]);
+    };
+    // The trajectories that can end inside chunk `k` are [c_lo, c_hi]: c_lo holds a token at or below the chunk's
+    // first, c_hi one at or above its last.  Values that are no trajectory (only with inconsistent lengths, which
+    // the preparation flags) are pulled into range.
+    auto cand_lo = [&](int k) -> int {
+      const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+      const int c = __ldcg(a.ws.chunk_first + (max(p0, t_lo) / kAdvChunk));
+      return c < 0 ? 0 : (c > a.B ? a.B : c);
+    };
+    auto cand_hi = [&](int k) -> int {
+      const long long p_end = min(t_hi - (long long)k * kAdvChunk, a.total);
+      const long long g = (p_end - 1) / kAdvChunk + 1;
+      if (g >= a.nchunks) return a.B - 1;
+      const int c = __ldcg(a.ws.chunk_first + g);
+      return c < 0 ? -1 : (c >= a.B ? a.B - 1 : c);
+    };
+    struct Traj { long long o0, o1; unsigned st; };
+    auto traj_load = [&](int i, int c_hi) -> Traj {
+      Traj t{0, 0, 0u};
+      if (i <= c_hi) {
+        t.o0 = __ldcg(a.ws.offsets + i);
+        t.o1 = __ldcg(a.ws.offsets + i + 1);
+        t.st = a.stopped[i];
+      }
+      return t;
+    };
+    auto traj_mark = [&](int k, const Traj& t) {
+      const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+      const long long p_lo = max(p0, t_lo);
+      const long long p_end = min(p0 + kAdvChunk, a.total);
+      if (t.o1 > t.o0 && t.o1 - 1 >= p_lo && t.o1 - 1 < p_end) {
+        const int pos = (int)(t.o1 - 1 - p0);
+        atomicOr(fwbuf + (k % kAdvStages) * kAdvThreads + (pos >> 4), (1u | (t.st ? 0x10000u : 0u)) << (pos & 15));
+      }
+    };
+
+    const int pre = nck < kAdvStages ? nck : kAdvStages;
+    if (lane == 0)
+      for (int k = 0; k < pre; ++k) issue_copies(k);       // needs nothing of the preparation kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // everything below reads what it wrote
+    int c_lo = cand_lo(0), c_hi = cand_hi(0);               // candidates of the chunk in hand
+    int n_lo = nck > 1 ? cand_lo(1) : 0, n_hi = nck > 1 ? cand_hi(1) : -1;   // and of the next one
+    Traj t0 = traj_load(c_lo + lane, c_hi);                 // the lane's first candidate, loaded one chunk ahead
+    for (int k = 0; k < nck; ++k) {
+      const int stage = k % kAdvStages;
+      if (k >= kAdvStages) {
+        if (!mbar_wait_bounded(&empty[stage], (uint32_t)((k / kAdvStages - 1) & 1), nullptr)) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
+        if (lane == 0) issue_copies(k);
+      }
+      traj_mark(k, t0);
+      for (int i = c_lo + 32 + lane; i <= c_hi; i += 32) traj_mark(k, traj_load(i, c_hi));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&full[stage]);             // the flags (and lane 0's ordinary stores) are in place
+      c_lo = n_lo; c_hi = n_hi;
+      t0 = traj_load(c_lo + lane, c_hi);
+      if (k + 2 < nck) { n_lo = cand_lo(k + 2); n_hi = cand_hi(k + 2); }
+      else { n_lo = 0; n_hi = -1; }
     }
-  };
+    return;
+  }
 
-  uint32_t phase[2] = {0u, 0u};
+  // =============================== scanning warps ===============================
   unsigned last_mask = 0;
   double d[kAdvPerThread];
   Map m, after;
 
-  // Waits for `stage`, folds the chunk `k` it holds: leaves the thread's TD errors in d[], its end mask in
-  // last_mask, its own map in m and the map of everything after the thread inside the chunk in `after`; the
-  // stage's flag bytes are cleared for their next use.  Contains one __syncthreads().
-  auto fold = [&](int k, int stage, int par) {
+  // Waits for chunk `k`, folds it: leaves the thread's TD errors in d[], its end mask in last_mask, its own map in
+  // m and the map of everything after the thread inside the chunk in `after`; the thread's flag word is cleared
+  // and the stage handed back to the producer as soon as the thread has read its part.  Contains one rendezvous
+  // of the scanning warps.
+  auto fold = [&](int k) {
+    const int stage = k % kAdvStages;
+    const int par = k & 1;
     const float* rs = rbuf + stage * kAdvChunk;
     const float* vs = vbuf + stage * kAdvVStride;
     const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
-    if (!mbar_wait_bounded(&mbar[stage], phase[stage], nullptr)) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
-    phase[stage] ^= 1u;
+    if (!mbar_wait_bounded(&full[stage], (uint32_t)((k / kAdvStages) & 1), nullptr)) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
     float r[kAdvPerThread], v[kAdvPerThread];
 #pragma unroll
     for (int h = 0; h < kAdvPerThread / 4; ++h) {
@@ -242,17 +307,12 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
       v[4 * h] = vv.x; v[4 * h + 1] = vv.y; v[4 * h + 2] = vv.z; v[4 * h + 3] = vv.w;
     }
     const float v_after = vs[q0 + kAdvPerThread];   // the next thread's first value; for the last thread, the next chunk's
-    uint4* fp = reinterpret_cast<uint4*>(flagbuf + stage * kAdvChunk) + tid;
-    const uint4 f16 = *fp;
-    *fp = make_uint4(0u, 0u, 0u, 0u);
-    const unsigned fw[4] = {f16.x, f16.y, f16.z, f16.w};
-    unsigned fail_mask = 0;
-    last_mask = 0;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {   // gather bit 0 (resp. bit 1) of four bytes into four adjacent bits
-      last_mask |= (((fw[w] & 0x01010101u) * 0x01020408u) >> 24) << (4 * w);
-      fail_mask |= ((((fw[w] >> 1) & 0x01010101u) * 0x01020408u) >> 24) << (4 * w);
-    }
+    uint32_t* fp = fwbuf + stage * kAdvThreads + tid;
+    const uint32_t fw = *fp;
+    *fp = 0u;
+    mbar_arrive(&empty[stage]);                     // release: this thread's reads and its cleared flag word come first
+    last_mask = fw & 0xffffu;
+    unsigned fail_mask = fw >> 16;
     {
       // the array's very last token ends a trajectory even if the lengths are inconsistent
       const long long e_last = a.total - 1 - p0 - q0;
@@ -283,7 +343,7 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
         vd_next = vd;
       }
     }
-    // Tokens past the end of the array (only in its last chunk) read as zeros; the array's last token is a
+    // Tokens past the end of the array (at most three, in its last chunk) read as zeros; the array's last token is a
     // forced trajectory end, so nothing of them reaches a stored result.
     m = Map{last_mask ? 0.0 : pw[kAdvPerThread], mb};   // X survives the thread only if no trajectory ends in it
     Map inc = m;   // inclusive suffix inside the warp
@@ -295,31 +355,11 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
     if (lane == 0) warp_agg[par][warp] = inc;
     after = Map{shfl_down_d(inc.a, 1), shfl_down_d(inc.b, 1)};   // exclusive within the warp
     if (lane == 31) after = Map{1.0, 0.0};
-    __syncthreads();   // warp aggregates written; every thread has read its part of the stage
+    cta_rendezvous(kAdvThreads);   // warp aggregates written
     for (int w = warp + 1; w < kAdvWarps; ++w) after = compose(after, warp_agg[par][w]);
   };
 
-  if (tid == 0) {
-    halo_traj = -1;
-    mbar_init(&mbar[0], 1);
-    mbar_init(&mbar[1], 1);
-    mbar_init_fence();
-    double p = 1.0;
-    for (int i = 0; i <= kAdvPerThread; ++i) { pw[i] = p; p *= a.gl; }
-  }
-  reinterpret_cast<uint4*>(flagbuf)[tid] = make_uint4(0u, 0u, 0u, 0u);
-  reinterpret_cast<uint4*>(flagbuf)[tid + kAdvThreads] = make_uint4(0u, 0u, 0u, 0u);
-  __syncthreads();
-  if (nck <= 0) return;
-
-  // ---- the two highest chunks of the range are on their way while the CTA works out what follows the range ----
-  fetch(0, 1);
-  if (nck > 1) fetch(1, 0);
-  // Launched as a programmatic dependent of the preparation kernel: everything above overlaps with it, everything
-  // below reads what it wrote.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  mark_ends(0, 1);
-  if (nck > 1) mark_ends(1, 0);
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // everything below reads what the preparation kernel wrote
 
   // ---- the advantage of the token that follows the range (token t_hi).  Its trajectory continues in the next CTA's
   //      range; unrolled, Eq. 5 makes it the weighted sum of the rest of that one trajectory's TD errors,
@@ -327,22 +367,22 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
   //      served by L2): thread t owns tokens 4t .. 4t+3 of every 1024.  CTAs therefore never wait for one another. ----
   if (t_hi < a.total) {   // find the trajectory that holds token t_hi
     int first = __ldcg(a.ws.chunk_first + (t_hi / kAdvChunk));
-    if ((unsigned)first >= (unsigned)a.B) first = a.B;
+    if ((unsigned)first >= (unsigned)a.B) first = a.B;   // only with inconsistent lengths (flagged by the preparation)
     for (int i = first + tid; i < a.B; i += kAdvThreads) {
       const long long o0 = __ldcg(a.ws.offsets + i);
       const long long o1 = __ldcg(a.ws.offsets + i + 1);
+      const int st = a.stopped[i];
       if (o0 > t_hi) break;
-      if (o1 > t_hi) halo_traj = i;
+      if (o1 > t_hi) { halo_traj = i; halo_end = o1; halo_failed = st; }
     }
   }
-  __syncthreads();
+  cta_rendezvous(kAdvThreads);
   {
     double part = 0.0;
-    const int i = halo_traj;
-    if (i >= 0) {
-      const long long t_end = min(__ldcg(a.ws.offsets + i + 1), a.total);          // the trajectory's end
+    if (halo_traj >= 0) {
+      const long long t_end = min(halo_end, a.total);                              // the trajectory's end
       const long long end = (t_end - t_hi > a.halo_cap) ? t_hi + a.halo_cap : t_end; // the part whose weights matter
-      const bool failed = a.stopped[i] != 0;
+      const bool failed = halo_failed != 0;
       double wt = 1.0, sq = a.gl;                        // (gamma*lambda)^(4 tid) by binary powering
       for (unsigned ex = 4u * tid; ex; ex >>= 1) {
         if (ex & 1u) wt *= sq;
@@ -382,30 +422,29 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) part += shfl_down_d(part, o);
-    if (lane == 0) warp_agg[0][warp].b = part;
-    __syncthreads();
+    if (lane == 0) warp_agg[1][warp].b = part;             // chunk 0 uses warp_agg[0]
+    cta_rendezvous(kAdvThreads);
     if (tid == 0) {
       double carry = 0.0;                                  // past the end of the array the value is 0
-      for (int w = 0; w < kAdvWarps; ++w) carry += warp_agg[0][w].b;
-      carry_buf[1] = carry;
+      for (int w = 0; w < kAdvWarps; ++w) carry += warp_agg[1][w].b;
+      carry_buf[0] = carry;
     }
+    // chunk 0's rendezvous comes between this write and its readers, and between the reads of warp_agg[1] above and
+    // chunk 1's writes to it
   }
-  __syncthreads();   // carry, flags of both stages
 
-  // ---- the range, from its highest chunk down; chunk k sits in stage (k + 1) & 1 ----
-  int s = 1;
-  for (int k = 0; k < nck; ++k, s ^= 1) {
+  // ---- the range, from its highest chunk down ----
+  for (int k = 0; k < nck; ++k) {
+    const int par = k & 1;
     const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
     const int q_lo = (int)(max(p0, t_lo) - p0);                               // positions [q_lo, q_hi) hold this
     const int q_hi = (int)min((long long)kAdvChunk, a.total - p0);           // CTA's tokens
-    fold(k, s, s);
-    const double carry_in = carry_buf[s];
+    fold(k);
+    const double carry_in = carry_buf[par];
     if (tid == 0) {
       const Map whole = compose(m, after);
-      carry_buf[s ^ 1] = fma(whole.a, carry_in, whole.b);       // what follows the next (lower) chunk
+      carry_buf[par ^ 1] = fma(whole.a, carry_in, whole.b);     // what follows the next (lower) chunk
     }
-    // the stage is free: start the copy of the chunk two below, and mark its trajectory ends
-    if (k + 2 < nck) { fetch(k + 2, s); mark_ends(k + 2, s); }
 
     // ---- replay the thread's tokens with the value that follows them ----
     double x = fma(after.a, carry_in, after.b);
@@ -443,8 +482,8 @@ __global__ void __launch_bounds__(kAdvThreads, kAdvCtasPerSm) espo_adv_scan_kern
           if (a.ret) a.ret[p0 + q0 + e] = out[e] + __ldcs(a.values + p0 + q0 + e);
         }
     }
-    // No barrier here: the next chunk's flags, carry and data are read after the barrier inside its fold(), and
-    // the warp aggregates alternate between two buffers.
+    // No rendezvous here: the next chunk's carry is read after the rendezvous inside its fold(), and the warp
+    // aggregates alternate between two buffers.
   }
 }
 
@@ -464,7 +503,7 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
   if (grid > a.nchunks) grid = a.nchunks;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kAdvThreads);
+  cfg.blockDim = dim3(kAdvCtaThreads);
   cfg.dynamicSmemBytes = kAdvSmemBytes;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
