@@ -32,12 +32,15 @@
 namespace espo {
 
 constexpr int kAdvThreads = 256;                        // scanning threads
-constexpr int kAdvPerThread = 16;
-constexpr int kAdvChunk = kAdvThreads * kAdvPerThread;   // 4096 tokens
+// Tokens per scanning thread: a multiple of 4 (16-byte accesses), at most 16 (flag word), and an odd number of
+// 16-byte pieces, so that the threads' shared-memory rows (48 bytes apart) fall into different banks.
+constexpr int kAdvPerThread = 12;
+constexpr int kAdvChunk = kAdvThreads * kAdvPerThread;   // 3072 tokens
+static_assert(kAdvPerThread % 4 == 0 && kAdvPerThread <= 16, "flag word: 16 end bits and 16 stop bits");
 constexpr int kAdvWarps = kAdvThreads / 32;
 constexpr int kAdvCtaThreads = kAdvThreads + 32;          // the scanning threads and the producer warp
-constexpr int kAdvStages = 3;
-constexpr int kAdvCtasPerSm = 2;
+constexpr int kAdvStages = 2;
+constexpr int kAdvCtasPerSm = 3;
 constexpr int kMaxDevicesAdv = 64;
 constexpr int kPrepThreads = 1024;
 
@@ -253,7 +256,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
       const long long p_end = min(p0 + kAdvChunk, a.total);
       if (t.o1 > t.o0 && t.o1 - 1 >= p_lo && t.o1 - 1 < p_end) {
         const int pos = (int)(t.o1 - 1 - p0);
-        atomicOr(fwbuf + (k % kAdvStages) * kAdvThreads + (pos >> 4), (1u | (t.st ? 0x10000u : 0u)) << (pos & 15));
+        atomicOr(fwbuf + (k % kAdvStages) * kAdvThreads + (pos / kAdvPerThread), (1u | (t.st ? 0x10000u : 0u)) << (pos % kAdvPerThread));
       }
     };
 
@@ -322,7 +325,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     double mb = 0.0;
     double vd_next = (double)v_after;
     if (!__any_sync(kFullMask, last_mask != 0u)) {
-      // no trajectory ends among the warp's 512 tokens (the usual case): no per-token case distinctions
+      // no trajectory ends among the warp's tokens (the usual case): no per-token case distinctions
 #pragma unroll
       for (int e = kAdvPerThread - 1; e >= 0; --e) {
         const double vd = (double)v[e];
@@ -561,7 +564,7 @@ static int ensure_pool(int dev, int B, long long nchunks, AdvPool** out) {
 // trajectories and kNoAllocMaxChunks chunks.  Zero-filled when the module is loaded.
 // ---------------------------------------------------------------------------------------
 constexpr int kNoAllocMaxB = ESPO_NOALLOC_MAX_B;
-constexpr long long kNoAllocMaxChunks = (ESPO_NOALLOC_MAX_TOKENS + kAdvChunk - 1) / kAdvChunk;
+constexpr long long kNoAllocMaxChunks = ((ESPO_NOALLOC_MAX_TOKENS + kAdvChunk - 1) / kAdvChunk + 63) / 64 * 64;
 constexpr size_t kNaOffOffsets = 0;
 constexpr size_t kNaOffChunkFirst = kNaOffOffsets + ((8 * ((size_t)kNoAllocMaxB + 1) + 255) / 256) * 256;
 constexpr size_t kNaOffStatus = kNaOffChunkFirst + 4 * (size_t)kNoAllocMaxChunks;
