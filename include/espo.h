@@ -248,7 +248,7 @@ int espo_advantages_status(uint32_t* host_out, void* stream);
  * own pools at start-up, so that a cudaMalloc issued by a library fails; and a training loop
  * that cannot afford the device-wide synchronisation that cudaMalloc/cudaFree imply.  This call
  * never calls cudaMalloc, cudaFree or any other allocating routine: its scratch is a fixed
- * array of about 50 KB that is part of the library image, so every device that loads the
+ * array of about 55 KB that is part of the library image, so every device that loads the
  * library holds that array until the process exits.
  *
  * Arguments are those of espo_advantages, plus

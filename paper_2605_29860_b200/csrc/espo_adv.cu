@@ -1,23 +1,29 @@
 // TD errors and GAE over ragged, truncated trajectories (Eq. 4-5) with ESPO's absorbing
 // failure transition (Eq. 13), for sm_100a.
 //
-// The packed token array is cut into fixed chunks of kAdvChunk tokens regardless of where
-// trajectories begin and end, and every CTA of a persistent grid takes an equal, contiguous
-// range of chunks, so every CTA moves the same number of bytes (12 per token: reward and
-// value in, advantage out) whatever the length mix is.  Within a chunk the backward recursion
-// A_t = delta_t + k_t A_{t+1} (k_t = gamma*lambda, or 0 on a trajectory's last token) is a scan
-// over affine maps X -> b + a X: a thread folds its 16 consecutive tokens, the 256 threads'
-// maps are composed by a warp-shuffle suffix scan and a small cross-warp pass, all in double
-// precision (with gamma*lambda = 1 an advantage is a sum of up to 16k TD errors).  A CTA walks
-// its range from the highest chunk down and carries the value that follows a chunk in shared
-// memory.  The value that follows its highest chunk belongs to a trajectory that continues
-// in the next CTA's range: the CTA obtains it by folding (reading only) the rest of that one
-// trajectory first -- at most one trajectory's worth of extra reads per CTA, usually served by
-// L2 -- so CTAs never wait for one another.  Chunks reach shared memory through a two-stage
-// ring of bulk asynchronous copies (TMA without a tensor map) issued two chunks ahead.
+// Every CTA of a persistent grid takes an equal, contiguous range of the packed token array
+// (cut at multiples of four tokens, wherever trajectories begin and end), so every CTA moves the
+// same number of bytes (12 per token: reward and value in, advantage out) whatever the length
+// mix is, and walks it from the top down in chunks of kAdvChunk tokens.  Within a chunk the
+// backward recursion A_t = delta_t + k_t A_{t+1} (k_t = gamma*lambda, or 0 on a trajectory's
+// last token) is a scan over affine maps X -> b + a X: a thread folds its 12 consecutive tokens,
+// the 256 threads' maps are composed by a warp-shuffle suffix scan and a small cross-warp pass,
+// all in double precision (with gamma*lambda = 1 an advantage is a sum of up to 16k TD errors).
+// The value that follows a chunk is carried in shared memory.  The value that follows the
+// range belongs to a trajectory that continues in the next CTA's range: unrolled, Eq. 5 makes it
+// a weighted sum of the rest of that one trajectory's TD errors, which the CTA takes straight from
+// global memory first (read only, usually served by L2, and only as far as the weights
+// (gamma*lambda)^k can still matter) -- so CTAs never wait for one another.
 //
-// A small preparation kernel turns lengths into offsets and tells every chunk which
-// trajectory its first token belongs to.
+// The CTA is warp-specialised.  A producer warp keeps a ring of stages full with bulk asynchronous
+// copies (TMA without a tensor map) and turns the trajectory ends that fall into a chunk into one flag
+// word per scanning thread; the eight scanning warps touch global memory only to store results.  A
+// thread's 12 tokens are 48 bytes: consecutive threads' rows start in different shared-memory banks
+// (with 16 tokens, 64 bytes, every 128-bit read was a 4-way conflict per quarter warp).
+//
+// A small preparation kernel turns lengths into offsets and tells every kAdvChunk-th token which
+// trajectory it belongs to; the scan is launched as its programmatic dependent, so the ring fills
+// while the preparation still runs.
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>

@@ -41,7 +41,15 @@ def test_discount_variants(gamma, lam):
 
 
 @pytest.mark.parametrize("lengths", [[1], [2048], [2047], [2049], [4096, 4096], [1] * 5000, [0, 3, 0, 0, 2050, 0],
-                                     [70000], [2048, 1, 2047, 4097, 5], [3, 2045, 2048, 2048, 1]])
+                                     [70000], [2048, 1, 2047, 4097, 5], [3, 2045, 2048, 2048, 1],
+                                     # around the kernel's 3072-token chunks and its 4-token range granularity
+                                     [2], [3], [5], [3071], [3072], [3073], [3072, 3072], [3070, 3, 3071, 6145], [6143, 1, 0, 7],
+                                     # thousands of one- and two-token trajectories: more ends in a chunk than one round
+                                     # of the flag-setting warp covers, over several CTAs' ranges
+                                     [1] * 40001, [2, 1] * 9000 + [30000, 1, 1],
+                                     # one trajectory crossing many CTAs' ranges (each looks ahead to its end, or as
+                                     # far as the weights matter), then short ones
+                                     [1_500_002, 7, 1, 4099]])
 def test_edge_lengths(lengths):
     g = torch.Generator("cuda").manual_seed(len(lengths) + sum(lengths))
     L = torch.tensor(lengths, dtype=torch.int32, device="cuda")
