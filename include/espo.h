@@ -229,6 +229,20 @@ int espo_advantages_returns(const float* rewards, const float* values, const int
                             float gamma, float lambda, float r_fail, float* adv_out,
                             float* returns_out, void* stream);
 
+/* espo_advantages_returns that also leaves the two sums a trainer normalises ("whitens") a batch of advantages
+ * with.  The paper does not normalise advantages (Sec. 3 uses the GAE of Eq. 5 as it is); this is the usual
+ * PPO companion step, offered because the sums fall out of the same pass.
+ *   stats_out    device float64 [2], 8-byte aligned, or NULL (then exactly espo_advantages_returns):
+ *                stats_out[0] = sum_t A_t, stats_out[1] = sum_t A_t^2 over all total_tokens tokens, taken in
+ *                double precision before the advantages are rounded to float32; mean = stats_out[0] / total_tokens,
+ *                variance = stats_out[1] / total_tokens - mean^2.  With B == 0 or total_tokens == 0 both are set to 0.
+ * Every CTA adds up its own tokens and the CTA that finishes last adds up the CTAs' sums in a fixed order, so
+ * repeated calls on the same input give bit-identical sums.  Everything else as for espo_advantages. */
+int espo_advantages_stats(const float* rewards, const float* values, const int32_t* lengths,
+                          const uint8_t* stopped, int32_t B, int64_t total_tokens,
+                          float gamma, float lambda, float r_fail, float* adv_out,
+                          float* returns_out, double* stats_out, void* stream);
+
 /* Pre-size the advantage workspace of the current device so that later calls with
  * B <= max_B and total_tokens <= max_tokens allocate nothing. */
 int espo_advantages_reserve(int32_t max_B, int64_t max_tokens);

@@ -77,6 +77,7 @@ def lib():
         L.espo_end_batch.argtypes = [vp, f32, f32, f32, f32, f32, i32, C.POINTER(espo_params), C.POINTER(C.c_double), vp]
         L.espo_advantages.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp]
         L.espo_advantages_returns.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp]
+        L.espo_advantages_stats.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp, vp]
         L.espo_advantages_noalloc.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp]
         L.espo_advantages_reserve.argtypes = [i32, i64]
         L.espo_advantages_status.argtypes = [C.POINTER(C.c_uint32), vp]
@@ -85,7 +86,8 @@ def lib():
         L.espo_last_cuda_error.argtypes = []
         for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_state_view",
                   "espo_compact_active", "espo_state_status", "espo_end_batch", "espo_advantages", "espo_advantages_reserve",
-                  "espo_advantages_status", "espo_advantages_noalloc", "espo_advantages_returns", "espo_last_cuda_error"):
+                  "espo_advantages_status", "espo_advantages_noalloc", "espo_advantages_returns", "espo_advantages_stats",
+                  "espo_last_cuda_error"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -251,6 +253,33 @@ def espo_advantages_returns(rewards: torch.Tensor, values: torch.Tensor, lengths
                                          total, gamma, lam, r_fail, _dev_ptr(adv_out, "adv_out"),
                                          _dev_ptr(returns_out, "returns_out"), _stream(stream)),
            "espo_advantages_returns")
+
+
+def espo_advantages_stats(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.Tensor, stopped: torch.Tensor,
+                          gamma: float, lam: float, r_fail: float, adv_out: torch.Tensor, stats_out: torch.Tensor,
+                          returns_out: Optional[torch.Tensor] = None, total_tokens: Optional[int] = None,
+                          stream=None) -> None:
+    """espo_advantages_returns that also leaves sum A_t and sum A_t^2 in ``stats_out`` (float64 [2]); see ``espo.h``."""
+    for t, n, dt in ((rewards, "rewards", torch.float32), (values, "values", torch.float32),
+                     (adv_out, "adv_out", torch.float32), (lengths, "lengths", torch.int32),
+                     (stopped, "stopped", torch.uint8), (stats_out, "stats_out", torch.float64)) + \
+            (() if returns_out is None else ((returns_out, "returns_out", torch.float32),)):
+        if t.dtype != dt or not t.is_contiguous():
+            raise ValueError(f"{n} must be a contiguous {dt} tensor")
+    total = rewards.numel() if total_tokens is None else total_tokens
+    if values.numel() < total or adv_out.numel() < total or rewards.numel() < total or \
+            (returns_out is not None and returns_out.numel() < total):
+        raise ValueError("rewards, values and the outputs must hold total_tokens entries")
+    if stopped.numel() < lengths.numel():
+        raise ValueError("stopped is shorter than lengths")
+    if stats_out.numel() < 2:
+        raise ValueError("stats_out must hold two float64")
+    _check(lib().espo_advantages_stats(_dev_ptr(rewards, "rewards"), _dev_ptr(values, "values"),
+                                       _dev_ptr(lengths, "lengths"), _dev_ptr(stopped, "stopped"), lengths.numel(),
+                                       total, gamma, lam, r_fail, _dev_ptr(adv_out, "adv_out"),
+                                       _dev_ptr(returns_out, "returns_out"), _dev_ptr(stats_out, "stats_out"),
+                                       _stream(stream)),
+           "espo_advantages_stats")
 
 
 def espo_advantages(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.Tensor, stopped: torch.Tensor,

@@ -54,6 +54,8 @@ struct AdvWorkspace {
   long long* offsets;     // [B+1] exclusive prefix sum of lengths
   int* chunk_first;       // [nchunks] trajectory that owns the chunk's first token
   unsigned* status;       // sticky ESPO_DEV_* bits
+  double* partials;       // [2 * grid] per-CTA sums of A and A^2 (only with stats)
+  unsigned* done;         // CTAs that have written their partial sums; the last one resets it
 };
 
 struct AdvArgs {
@@ -63,6 +65,7 @@ struct AdvArgs {
   const uint8_t* stopped;
   float* adv;
   float* ret;             // optional: returns A_t + V_t (value targets), same layout as adv; may be null
+  double* stats;          // optional: [2] sum of A_t and of A_t^2 over all tokens; may be null
   int B;
   long long total;
   int nchunks;
@@ -160,6 +163,9 @@ constexpr size_t kAdvSmemBytes =
 
 // kAdvThreads threads scan; one more warp (the producer) keeps the ring full and sets the flag words, so that no
 // scanning warp ever waits for a load from global memory.
+// STATS: also the batch sums of A and A^2.  RET: also the returns A_t + V_t; the scanning threads then keep a stage
+// until they have stored, because they read the values from it a second time.
+template <bool STATS, bool RET>
 __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_kernel(const AdvArgs a) {
   extern __shared__ __align__(128) unsigned char adv_smem[];
   float* rbuf = reinterpret_cast<float*>(adv_smem);
@@ -173,6 +179,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
   __shared__ int halo_traj;                                  // trajectory that crosses the range's upper end, or -1,
   __shared__ long long halo_end;                             // its end offset
   __shared__ int halo_failed;                                // and whether it was stopped
+  __shared__ int is_last_cta;                                // statistics: this CTA adds up every CTA's partial sums
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const double r_fail_d = (double)a.r_fail;
@@ -200,9 +207,9 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
   }
   for (int i = tid; i < kAdvStages * kAdvThreads; i += kAdvCtaThreads) fwbuf[i] = 0u;
   __syncthreads();
-  if (nck <= 0) return;
 
   if (warp == kAdvWarps) {
+    if (nck <= 0) return;
     // =============================== producer warp ===============================
     // Starts the copies of chunk `k` (lane 0).  A chunk is two bulk copies (plus 16 bytes for the value after the
     // chunk) that complete on the stage's mbarrier; of a chunk that reaches past the end of the array (only the
@@ -319,7 +326,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     uint32_t* fp = fwbuf + stage * kAdvThreads + tid;
     const uint32_t fw = *fp;
     *fp = 0u;
-    mbar_arrive(&empty[stage]);                     // release: this thread's reads and its cleared flag word come first
+    if (!RET) mbar_arrive(&empty[stage]);           // release: this thread's reads and its cleared flag word come first
     last_mask = fw & 0xffffu;
     unsigned fail_mask = fw >> 16;
     {
@@ -374,7 +381,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
   //      range; unrolled, Eq. 5 makes it the weighted sum of the rest of that one trajectory's TD errors,
   //      sum_k (gamma*lambda)^k delta_k, which the CTA's threads take straight from global memory (read only, usually
   //      served by L2): thread t owns tokens 4t .. 4t+3 of every 1024.  CTAs therefore never wait for one another. ----
-  if (t_hi < a.total) {   // find the trajectory that holds token t_hi
+  if (nck > 0 && t_hi < a.total) {   // find the trajectory that holds token t_hi
     int first = __ldcg(a.ws.chunk_first + (t_hi / kAdvChunk));
     if ((unsigned)first >= (unsigned)a.B) first = a.B;   // only with inconsistent lengths (flagged by the preparation)
     for (int i = first + tid; i < a.B; i += kAdvThreads) {
@@ -443,6 +450,8 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
   }
 
   // ---- the range, from its highest chunk down ----
+  constexpr bool want_stats = STATS;
+  double sum_a = 0.0, sum_a2 = 0.0;   // of the advantages this thread stores (before rounding to float)
   for (int k = 0; k < nck; ++k) {
     const int par = k & 1;
     const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
@@ -458,27 +467,31 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     // ---- replay the thread's tokens with the value that follows them ----
     double x = fma(after.a, carry_in, after.b);
     float out[kAdvPerThread];
+    const bool whole_thread = (q0 >= q_lo && q0 + kAdvPerThread <= q_hi);
     if (!__any_sync(kFullMask, last_mask != 0u)) {
 #pragma unroll
       for (int e = kAdvPerThread - 1; e >= 0; --e) {
         x = fma(a.gl, x, d[e]);
         out[e] = (float)x;
+        if (want_stats && (whole_thread || (q0 + e >= q_lo && q0 + e < q_hi))) { sum_a += x; sum_a2 = fma(x, x, sum_a2); }
       }
     } else {
 #pragma unroll
       for (int e = kAdvPerThread - 1; e >= 0; --e) {
         x = ((last_mask >> e) & 1u) ? d[e] : fma(a.gl, x, d[e]);
         out[e] = (float)x;
+        if (want_stats && (whole_thread || (q0 + e >= q_lo && q0 + e < q_hi))) { sum_a += x; sum_a2 = fma(x, x, sum_a2); }
       }
     }
-    if (q0 >= q_lo && q0 + kAdvPerThread <= q_hi) {
+    if (whole_thread) {
 #pragma unroll
       for (int h = 0; h < kAdvPerThread / 4; ++h)
         __stcs(reinterpret_cast<float4*>(a.adv + p0 + q0) + h, make_float4(out[4 * h], out[4 * h + 1], out[4 * h + 2], out[4 * h + 3]));
-      if (a.ret) {   // the values were read a moment ago: this re-read is served by L2
+      if (RET) {
+        const float* vs = vbuf + (k % kAdvStages) * kAdvVStride;
 #pragma unroll
         for (int h = 0; h < kAdvPerThread / 4; ++h) {
-          const float4 vv = __ldcs(reinterpret_cast<const float4*>(a.values + p0 + q0) + h);
+          const float4 vv = *reinterpret_cast<const float4*>(vs + q0 + 4 * h);
           __stcs(reinterpret_cast<float4*>(a.ret + p0 + q0) + h,
                  make_float4(out[4 * h] + vv.x, out[4 * h + 1] + vv.y, out[4 * h + 2] + vv.z, out[4 * h + 3] + vv.w));
         }
@@ -488,11 +501,50 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
       for (int e = 0; e < kAdvPerThread; ++e)
         if (q0 + e >= q_lo && q0 + e < q_hi) {
           a.adv[p0 + q0 + e] = out[e];
-          if (a.ret) a.ret[p0 + q0 + e] = out[e] + __ldcs(a.values + p0 + q0 + e);
+          if (RET) a.ret[p0 + q0 + e] = out[e] + vbuf[(k % kAdvStages) * kAdvVStride + q0 + e];
         }
     }
+    if (RET) mbar_arrive(&empty[k % kAdvStages]);   // release: the second read of the values comes first
     // No rendezvous here: the next chunk's carry is read after the rendezvous inside its fold(), and the warp
     // aggregates alternate between two buffers.
+  }
+
+  // ---- optional batch sums of A and A^2: one pair per CTA, added up in a fixed order by whichever CTA finishes
+  //      last, so that repeated calls give bit-identical sums ----
+  if (want_stats) {
+    cta_rendezvous(kAdvThreads);            // the last chunk's readers of warp_agg are done
+#pragma unroll
+    for (int o = 16; o; o >>= 1) { sum_a += shfl_down_d(sum_a, o); sum_a2 += shfl_down_d(sum_a2, o); }
+    if (lane == 0) warp_agg[0][warp] = Map{sum_a, sum_a2};
+    cta_rendezvous(kAdvThreads);
+    if (tid == 0) {
+      double t1 = 0.0, t2 = 0.0;
+      for (int w = 0; w < kAdvWarps; ++w) { t1 += warp_agg[0][w].a; t2 += warp_agg[0][w].b; }
+      a.ws.partials[2 * blockIdx.x] = t1;
+      a.ws.partials[2 * blockIdx.x + 1] = t2;
+      __threadfence();                      // the partial sums are visible before the count moves
+      is_last_cta = (atomicAdd(a.ws.done, 1u) == gridDim.x - 1);
+    }
+    cta_rendezvous(kAdvThreads);
+    if (is_last_cta) {
+      __threadfence();
+      double t1 = 0.0, t2 = 0.0;
+      for (unsigned b = tid; b < gridDim.x; b += kAdvThreads) {
+        t1 += __ldcg(a.ws.partials + 2 * b);
+        t2 += __ldcg(a.ws.partials + 2 * b + 1);
+      }
+#pragma unroll
+      for (int o = 16; o; o >>= 1) { t1 += shfl_down_d(t1, o); t2 += shfl_down_d(t2, o); }
+      if (lane == 0) warp_agg[1][warp] = Map{t1, t2};
+      cta_rendezvous(kAdvThreads);
+      if (tid == 0) {
+        double u1 = 0.0, u2 = 0.0;
+        for (int w = 0; w < kAdvWarps; ++w) { u1 += warp_agg[1][w].a; u2 += warp_agg[1][w].b; }
+        a.stats[0] = u1;
+        a.stats[1] = u2;
+        *a.ws.done = 0u;                    // ready for the next call
+      }
+    }
   }
 }
 
@@ -502,8 +554,10 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
   int dev = 0;
   ESPO_CUDA_TRY(cudaGetDevice(&dev));
   if (dev >= 0 && dev < kMaxDevicesAdv && !attr_set[dev]) {
-    ESPO_CUDA_TRY(cudaFuncSetAttribute((const void*)espo_adv_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)kAdvSmemBytes));
+    const void* variants[4] = {(const void*)espo_adv_scan_kernel<false, false>, (const void*)espo_adv_scan_kernel<false, true>,
+                               (const void*)espo_adv_scan_kernel<true, false>, (const void*)espo_adv_scan_kernel<true, true>};
+    for (const void* f : variants)
+      ESPO_CUDA_TRY(cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAdvSmemBytes));
     attr_set[dev] = true;
   }
   espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
@@ -520,7 +574,10 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel, a));
+  if (a.stats && a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<true, true>, a));
+  else if (a.stats) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<true, false>, a));
+  else if (a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, true>, a));
+  else ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, false>, a));
   return ESPO_OK;
 }
 
@@ -551,13 +608,15 @@ static int ensure_pool(int dev, int B, long long nchunks, AdvPool** out) {
     }
     size_t off = 0;
     auto carve = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    const size_t o_off = carve(8 * ((size_t)nb + 1)), o_cf = carve(4 * (size_t)nc), o_st = carve(4);
     if (!p.sm_count) ESPO_CUDA_TRY(cudaDeviceGetAttribute(&p.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    const size_t o_off = carve(8 * ((size_t)nb + 1)), o_cf = carve(4 * (size_t)nc), o_st = carve(4);
+    const size_t o_pa = carve(16 * (size_t)p.sm_count * kAdvCtasPerSm), o_dn = carve(4);
     ESPO_CUDA_TRY(cudaMalloc(&p.arena, off));
     ESPO_CUDA_TRY(cudaMemset(p.arena, 0, off));
     unsigned char* b = static_cast<unsigned char*>(p.arena);
     p.ws.offsets = (long long*)(b + o_off); p.ws.chunk_first = (int*)(b + o_cf);
     p.ws.status = (unsigned*)(b + o_st);
+    p.ws.partials = (double*)(b + o_pa); p.ws.done = (unsigned*)(b + o_dn);
     p.cap_B = nb; p.cap_chunks = nc;
   }
   *out = &p;
@@ -620,6 +679,7 @@ int espo_advantages_noalloc(const float* rewards, const float* values, const int
   // kernel rewrites every offset and chunk owner this call reads, and the built-in status word is only OR-ed into.
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = nullptr;
+  a.stats = nullptr; a.ws.partials = nullptr; a.ws.done = nullptr;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
   set_discount(a, gamma, lambda);
   a.r_fail = r_fail;
@@ -639,12 +699,16 @@ int espo_advantages_reserve(int32_t max_B, int64_t max_tokens) {
   return ensure_pool(dev, max_B, (max_tokens + kAdvChunk - 1) / kAdvChunk, &p);
 }
 
-int espo_advantages_returns(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
-                            int32_t B, int64_t total_tokens, float gamma, float lambda, float r_fail, float* adv_out,
-                            float* returns_out, void* stream) {
+int espo_advantages_stats(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
+                          int32_t B, int64_t total_tokens, float gamma, float lambda, float r_fail, float* adv_out,
+                          float* returns_out, double* stats_out, void* stream) {
   using namespace espo;
   if (B < 0 || total_tokens < 0) return ESPO_ERR_BAD_SHAPE;
-  if (B == 0 || total_tokens == 0) return ESPO_OK;
+  if ((uintptr_t)stats_out % 8) return ESPO_ERR_ALIGN;
+  if (B == 0 || total_tokens == 0) {
+    if (stats_out) ESPO_CUDA_TRY(cudaMemsetAsync(stats_out, 0, 2 * sizeof(double), (cudaStream_t)stream));
+    return ESPO_OK;
+  }
   if (!rewards || !values || !lengths || !stopped || !adv_out) return ESPO_ERR_NULL;
   if (((uintptr_t)rewards % 16) || ((uintptr_t)values % 16) || ((uintptr_t)adv_out % 16) || ((uintptr_t)lengths % 4) ||
       ((uintptr_t)returns_out % 16))
@@ -661,11 +725,19 @@ int espo_advantages_returns(const float* rewards, const float* values, const int
   cudaStream_t s = (cudaStream_t)stream;
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = returns_out;
+  a.stats = stats_out;
   a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
   set_discount(a, gamma, lambda);
   a.r_fail = r_fail;
   a.ws = p->ws;
   return launch_advantages(a, p->sm_count, s);
+}
+
+int espo_advantages_returns(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
+                            int32_t B, int64_t total_tokens, float gamma, float lambda, float r_fail, float* adv_out,
+                            float* returns_out, void* stream) {
+  return espo_advantages_stats(rewards, values, lengths, stopped, B, total_tokens, gamma, lambda, r_fail, adv_out,
+                               returns_out, nullptr, stream);
 }
 
 int espo_advantages(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,

@@ -115,3 +115,36 @@ def test_returns_are_written_in_the_same_pass():
                 togo = np.cumsum(seg[::-1])[::-1]
                 assert np.allclose(got[off[i]:off[i + 1]], togo, rtol=1e-4, atol=2e-5)
     assert espo.espo_advantages_status() == 0
+
+
+def test_batch_sums_come_out_of_the_same_pass():
+    # sum A and sum A^2 over all tokens, as a trainer needs them to normalise a batch of advantages
+    for seed, B, hi in ((9, 300, 9000), (10, 1024, 16384), (11, 3, 5)):
+        r, v, L, s = synth.ragged_trajectories(B, len_lo=1, len_hi=hi, seed=seed)
+        adv, ret = torch.empty_like(r), torch.empty_like(r)
+        stats = torch.full((2,), float("nan"), dtype=torch.float64, device="cuda")
+        espo.espo_advantages_stats(r, v, L, s, 1.0, 0.95, -1.0, adv, stats, returns_out=ret)
+        torch.cuda.synchronize()
+        assert espo.espo_advantages_status() == 0
+        # the C ABI takes lambda as float32: the oracle gets the same number
+        ref = oracle.advantages(r.cpu().numpy(), v.cpu().numpy(), L.cpu().numpy(), s.cpu().numpy(), 1.0,
+                                float(np.float32(0.95)), -1.0)
+        got = stats.cpu().numpy()
+        assert abs(got[0] - ref.sum()) <= 1e-9 * np.abs(ref).sum() + 1e-12
+        assert abs(got[1] - (ref * ref).sum()) <= 1e-9 * (ref * ref).sum() + 1e-12
+        assert np.all(np.abs(adv.cpu().numpy() - ref) <= 1e-5 + 1e-4 * np.abs(ref))
+        assert np.all(np.abs(ret.cpu().numpy() - (ref + v.cpu().numpy())) <= 2e-5 + 1e-4 * np.abs(ref + v.cpu().numpy()))
+        # a second call: bit-identical sums, and the plain entry point still gives the same advantages
+        stats2 = torch.zeros(2, dtype=torch.float64, device="cuda")
+        adv2 = torch.empty_like(r)
+        espo.espo_advantages_stats(r, v, L, s, 1.0, 0.95, -1.0, adv2, stats2)
+        adv3 = torch.empty_like(r)
+        espo.espo_advantages(r, v, L, s, 1.0, 0.95, -1.0, adv3)
+        torch.cuda.synchronize()
+        assert torch.equal(stats, stats2) and torch.equal(adv, adv2) and torch.equal(adv, adv3)
+    empty = torch.full((2,), 7.0, dtype=torch.float64, device="cuda")
+    z = torch.empty(0, device="cuda")
+    espo.espo_advantages_stats(z, z, torch.empty(0, dtype=torch.int32, device="cuda"),
+                               torch.empty(0, dtype=torch.uint8, device="cuda"), 1.0, 0.95, -1.0, z, empty)
+    torch.cuda.synchronize()
+    assert empty.tolist() == [0.0, 0.0]
