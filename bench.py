@@ -337,7 +337,37 @@ def main():
             "roofline": {"bound": "hbm", "achieved": adv_gbs, "peak": peak, "unit": "GB/s", "frac": adv_gbs / peak,
                          "traffic": None, "bytes_per_token": 12},
         }
+        ADV_TOKENS_NOMINAL = n_tok
         del r, v, L, s, a_out
+
+        # ---- library operations that move the same number of bytes, timed the same way: at these sizes (one launch
+        #      of 100-160 MB) launch, ramp and tail keep even a plain copy well below the large-buffer copy bandwidth
+        #      that `peak` is ----
+        if not args.no_sweep:
+            def time_us(fn, reps=100):
+                for i in range(5):
+                    fn(i)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(reps):
+                    fn(i)
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) * 1e3 / reps
+            half = [torch.empty(B // 2, V, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+            row_max = torch.empty(B, dtype=torch.bfloat16, device=dev)
+            adv_src = torch.empty(int(12.0 * ADV_TOKENS_NOMINAL / 8), dtype=torch.float32, device=dev).normal_()
+            adv_dst = torch.empty_like(adv_src)
+            lib = {
+                "copy_moving_step_bytes_us": time_us(lambda i: half[i % 2].copy_(bufs[i % N_BUFFERS][:B // 2])),
+                "torch_amax_over_step_logits_us": time_us(lambda i: torch.amax(bufs[i % N_BUFFERS], dim=1, out=row_max)),
+                "copy_moving_advantage_bytes_us": time_us(lambda i: adv_dst.copy_(adv_src)),
+                "note": f"step launch: {bytes_per_launch / 1e6:.1f} MB read; copy: {bytes_per_launch / 2e6:.1f} MB read + as much "
+                        f"written; advantage pass: {12.0 * ADV_TOKENS_NOMINAL / 1e6:.1f} MB moved",
+            }
+            out["library_ops_same_bytes"] = lib
+            del half, adv_src, adv_dst
 
         # ---- single-step bandwidth at other shapes (the large-batch sweep; rotating buffers larger than 2x L2) ----
         if not args.no_sweep:

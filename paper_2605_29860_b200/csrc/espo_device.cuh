@@ -152,6 +152,16 @@ __device__ __forceinline__ float expo_from_word(uint32_t word) {
   return -logf(u);
 }
 
+// ln E of an exponential draw E = -ln u in [6e-8, 17]: the Gumbel is -ln E.  E itself comes from the precise
+// logf (u close to 1 makes E tiny, and its relative accuracy is what the large Gumbels rest on); its logarithm
+// may be lg2.approx: absolute error below 2^-22 for E in (0.5, 2), relative error below 2^-22 elsewhere, i.e.
+// below 6e-6 at the far ends and below 1e-6 typically -- two orders under the sampler's tie margin.
+__device__ __forceinline__ float ln_expo(float e) {
+  float y;
+  asm("lg2.approx.f32 %0, %1;" : "=f"(y) : "f"(e));
+  return y * 0.6931471805599453f;
+}
+
 // Which Philox stream a draw belongs to: (step, slot, batch|level) are counter words 1..3.
 struct DrawStream {
   uint32_t k0, k1;     // seed halves
@@ -191,15 +201,18 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // Argmax of (score, index) over the warp; the lower index wins equal scores.  Lanes with
-// nothing to offer pass index < 0.  Every lane gets the result.
+// nothing to offer pass index < 0.  Every lane gets the result.  Scores are never NaN here.
+// Two warp-wide reductions in hardware: the largest offered score, then the smallest index
+// among the lanes that offer it.
 __device__ __forceinline__ void warp_argmax(float& score, int& index) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float s2 = __shfl_xor_sync(kFullMask, score, o);
-    const int i2 = __shfl_xor_sync(kFullMask, index, o);
-    const bool take = (i2 >= 0) && (index < 0 || s2 > score || (s2 == score && i2 < index));
-    if (take) { score = s2; index = i2; }
-  }
+  const float offered = index >= 0 ? score : __int_as_float(0xff800000);
+  float best;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(best) : "f"(offered));
+  const int cand = (index >= 0 && score == best) ? index : 0x7fffffff;
+  int first;
+  asm volatile("redux.sync.min.s32 %0, %1, 0xffffffff;" : "=r"(first) : "r"(cand));
+  score = best;
+  index = first == 0x7fffffff ? -1 : first;
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {

@@ -336,7 +336,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       const int id = __float_as_int(r.w);
       if (id >= 0 && (best_i < 0 || sc > best)) { best = sc; best_i = id; }
     } else {
-      const float ln_e = noise ? noise[b] : logf(expo_at(ds, 2u, (uint32_t)b));
+      const float ln_e = noise ? noise[b] : ln_expo(expo_at(ds, 2u, (uint32_t)b));
       const float sc = fmaf(m_b, a.inv_temp, log_sum(s_b) - ln_e);
       if (best_i < 0 || sc > best) { best = sc; best_i = b; }
     }
@@ -387,7 +387,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
     }
     run_m = mm;
     run_s = warp_sum(run_s);
-    run_u = warp_sum(run_u);
+    if (a.want_entropy) run_u = warp_sum(run_u);
   }
   const float M = run_m, S = run_s;
   const float log_S = logf(S);   // needed at the very end; started before the loads below
@@ -429,7 +429,7 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
     }
 
     // the sub-block's noise does not depend on the data: drawn while the loads above are in flight
-    const float ln_e1 = a.greedy ? 0.f : logf(expo_at(ds, 1u, (uint32_t)(sub_lo >> 5)));   // index = global sub-block number
+    const float ln_e1 = a.greedy ? 0.f : ln_expo(expo_at(ds, 1u, (uint32_t)(sub_lo >> 5)));   // index = global sub-block number
     if (a.greedy) {
       // first id equal to the maximum
       int first = -1;
@@ -452,18 +452,12 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       }
       warp_argmax(sc, j);
       const int sub_pick = max(j, blk_lo >> 5);        // j < 0 cannot happen: the block has a finite id
-      // ---- ids of the chosen sub-block: lane e takes id 32*sub_pick + e from the owning lane's registers ----
-      const int src = sub_pick & 31;
-      float mine = NINF;
-#pragma unroll
-      for (int i = 0; i < kSubIds; ++i) {
-        const float tv = __shfl_sync(kFullMask, x[i], src);
-        if (lane == i) mine = tv;
-      }
+      // ---- ids of the chosen sub-block: lane e takes id 32*sub_pick + e ----
       const int id = sub_pick * kSubIds + lane;
+      const float mine = (id < a.V) ? load_logit<ES>(row_base, id) : NINF;   // the lines are in L1 since the loads above
       float sc0 = NINF;
       int cand = -1;
-      if (id < a.V && mine > NINF) { sc0 = fmaf(mine, a.inv_temp, -logf(expo_at(ds, 0u, (uint32_t)id))); cand = id; }
+      if (id < a.V && mine > NINF) { sc0 = fmaf(mine, a.inv_temp, -ln_expo(expo_at(ds, 0u, (uint32_t)id))); cand = id; }
       warp_argmax(sc0, cand);
       token = max(cand, sub_pick * kSubIds);           // cand < 0 cannot happen for a sub-block with a finite id
       l_tok = __shfl_sync(kFullMask, mine, token & 31);
@@ -636,7 +630,7 @@ __device__ void prepare_rows(const StepArgs& a, const CtaRange& cr, const RowTab
         const uint32_t wd[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          if (b0 + i < a.nblk) tb.noise[(size_t)k * a.nblk + b0 + i] = logf(expo_from_word(wd[i]));
+          if (b0 + i < a.nblk) tb.noise[(size_t)k * a.nblk + b0 + i] = ln_expo(expo_from_word(wd[i]));
       }
     }
     __syncwarp();
