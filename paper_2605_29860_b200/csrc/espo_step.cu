@@ -322,38 +322,22 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
   int best_i = -1;            // HIER / greedy: block number; FLAT: token id
   bool poisoned = false;
   float run_m = NINF, run_s = 0.f, run_u = 0.f;   // sums of e and of e*t over this lane's blocks, relative to run_m
-  auto load_rec = [&](int b) -> float4 {
-    const float4* rp = static_cast<const float4*>(rec_row) + b;
-    return rec_local ? *rp : __ldcg(rp);       // shared-memory table, or global records written by other CTAs
-  };
-  auto score = [&](int b, const float4& r) {
-    const float m_b = r.x, s_b = r.y;
-    if (!(s_b > 0.f)) return;                   // all -inf block
-    if (a.greedy) {
-      if (m_b > best) { best = m_b; best_i = b; }                 // lowest block holding the maximum
-    } else if (SAMPLER == ESPO_SAMPLER_FLAT) {
-      const float sc = fmaf(m_b, a.inv_temp, r.z);                // the block's best, moved to the absolute scale
-      const int id = __float_as_int(r.w);
-      if (id >= 0 && (best_i < 0 || sc > best)) { best = sc; best_i = id; }
-    } else {
-      const float ln_e = noise ? noise[b] : ln_expo(expo_at(ds, 2u, (uint32_t)b));
-      const float sc = fmaf(m_b, a.inv_temp, log_sum(s_b) - ln_e);
-      if (best_i < 0 || sc > best) { best = sc; best_i = b; }
-    }
-  };
+  // The pass is one warp's latency chain for every row, so it is written without data-dependent branches: the five
+  // records of a lane are loaded, summed and scored as five independent strands.
   constexpr int kPerLane = 5;                   // records a lane holds at once (covers V <= 163840 in one go)
   for (int base = 0; base < a.nblk; base += 32 * kPerLane) {
     float4 r[kPerLane];
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i) {
       const int b = base + 32 * i + lane;
-      r[i] = (b < a.nblk) ? load_rec(b) : make_float4(NINF, 0.f, NINF, __int_as_float(-1));
+      // shared-memory table or global records written by other CTAs: one generic load that bypasses L1 serves both
+      r[i] = (b < a.nblk) ? ld_volatile_f4(static_cast<const float4*>(rec_row) + b) : make_float4(NINF, 0.f, NINF, __int_as_float(-1));
     }
     float lm = run_m;
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i) {
       poisoned |= !(r[i].y >= 0.0f) || isinf(r[i].y);   // NaN or inf sum: the block held NaN or +inf
-      if (r[i].y > 0.f) lm = fmaxf(lm, r[i].x);
+      lm = (r[i].y > 0.f) ? fmaxf(lm, r[i].x) : lm;
     }
     // sum of s_b 2^((m_b - lm) k2), independent terms; the carried sums are rescaled once.  Moving the reference
     // from R to R' turns (S, U) into f (S, U + (R - R') k2 S) with f = 2^((R - R') k2).
@@ -364,15 +348,55 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       acc = f * run_s;
     }
 #pragma unroll
-    for (int i = 0; i < kPerLane; ++i)
-      if (r[i].y > 0.f) {
-        const float dt = (r[i].x - lm) * a.k2, f = ex2_approx(dt);
-        acc = fmaf(r[i].y, f, acc);
-        if (SAMPLER == ESPO_SAMPLER_HIER) accu = fmaf(f, fmaf(dt, r[i].y, r[i].z), accu);
-      }
+    for (int i = 0; i < kPerLane; ++i) {
+      const bool ok = r[i].y > 0.f;
+      const float dt = ok ? (r[i].x - lm) * a.k2 : 0.f, f = ex2_approx(dt);
+      acc = ok ? fmaf(r[i].y, f, acc) : acc;
+      if (SAMPLER == ESPO_SAMPLER_HIER) accu = ok ? fmaf(f, fmaf(dt, r[i].y, r[i].z), accu) : accu;
+    }
     run_m = lm; run_s = acc; run_u = accu;
+    if (a.greedy) {
 #pragma unroll
-    for (int i = 0; i < kPerLane; ++i) score(base + 32 * i + lane, r[i]);
+      for (int i = 0; i < kPerLane; ++i) {
+        const bool take = (r[i].y > 0.f) && (r[i].x > best);          // lowest block holding the maximum
+        best = take ? r[i].x : best;
+        best_i = take ? base + 32 * i + lane : best_i;
+      }
+    } else if (SAMPLER == ESPO_SAMPLER_FLAT) {
+#pragma unroll
+      for (int i = 0; i < kPerLane; ++i) {
+        const float sc = fmaf(r[i].x, a.inv_temp, r[i].z);            // the block's best, moved to the absolute scale
+        const int id = __float_as_int(r[i].w);
+        const bool take = (r[i].y > 0.f) && id >= 0 && (best_i < 0 || sc > best);
+        best = take ? sc : best;
+        best_i = take ? id : best_i;
+      }
+    } else {
+      float ln_e[kPerLane];
+      if (noise) {
+#pragma unroll
+        for (int i = 0; i < kPerLane; ++i) {
+          const int b = base + 32 * i + lane;
+          ln_e[i] = (b < a.nblk) ? noise[b] : 0.f;
+        }
+      } else {
+        // the finalizer warp had not prepared this row's block-level noise: draw it here (kept as a loop: it is rare)
+#pragma unroll 1
+        for (int i = 0; i < kPerLane; ++i) {
+          const int b = base + 32 * i + lane;
+          const float e = (b < a.nblk) ? ln_expo(expo_at(ds, 2u, (uint32_t)b)) : 0.f;
+#pragma unroll
+          for (int j = 0; j < kPerLane; ++j) if (j == i) ln_e[j] = e;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kPerLane; ++i) {
+        const float sc = fmaf(r[i].x, a.inv_temp, log_sum(r[i].y) - ln_e[i]);
+        const bool take = (r[i].y > 0.f) && (best_i < 0 || sc > best);
+        best = take ? sc : best;
+        best_i = take ? base + 32 * i + lane : best_i;
+      }
+    }
   }
   {
     const float mm = warp_max(run_m);
