@@ -251,6 +251,22 @@ int espo_advantages_reserve(int32_t max_B, int64_t max_tokens);
  * of the current device to *host_out and clear it.  Synchronises `stream`. */
 int espo_advantages_status(uint32_t* host_out, void* stream);
 
+/* espo_advantages_returns for the padded layout: rewards, values and the outputs are [B, t_max] row-major and
+ * trajectory i owns the first lengths[i] entries of row i (Eq. 4-5 and 13 as for espo_advantages; the layout is this
+ * library's, the paper does not fix one).
+ *   rewards, values  device float32 [B * t_max], 16-byte aligned; what the padding holds is never used (it may be
+ *                    NaN)
+ *   lengths          device int32 [B], 0 <= lengths[i] <= t_max; a value outside sets ESPO_DEV_BAD_LENGTHS and is
+ *                    clamped
+ *   adv_out          device float32 [B * t_max]; padding entries are written as 0
+ *   returns_out      device float32 [B * t_max] or NULL; padding entries are written as 0
+ * The pass reads and writes all B * t_max entries (12 bytes each, 16 with returns), padding included; a batch that is
+ * mostly padding is cheaper packed.  Workspace and errors as for espo_advantages. */
+int espo_advantages_padded(const float* rewards, const float* values, const int32_t* lengths,
+                           const uint8_t* stopped, int32_t B, int32_t t_max,
+                           float gamma, float lambda, float r_fail, float* adv_out,
+                           float* returns_out, void* stream);
+
 /* Limits of espo_advantages_noalloc. */
 #define ESPO_NOALLOC_MAX_B       4096          /* trajectories per call                          */
 #define ESPO_NOALLOC_MAX_TOKENS  16777216      /* sum(lengths) per call (2^24)                   */

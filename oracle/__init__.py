@@ -209,6 +209,21 @@ def advantages(rewards, values, lengths, stopped, gamma, lam, r_fail, direct=Fal
     return out
 
 
+def advantages_padded(rewards, values, lengths, stopped, gamma, lam, r_fail, direct=False) -> np.ndarray:
+    """The same pass on a padded batch: ``rewards`` and ``values`` are [B, t_max], trajectory i owns the first
+    ``lengths[i]`` entries of row i (Eq. 4-5, 13 row by row).  Padding is never read (NaN there is fine) and comes
+    back as 0."""
+    r = np.asarray(rewards, dtype=np.float64)
+    v = np.asarray(values, dtype=np.float64)
+    L = np.asarray(lengths, dtype=np.int32)
+    B, t_max = r.shape
+    assert v.shape == r.shape and L.size == B and np.all((L >= 0) & (L <= t_max))
+    valid = np.arange(t_max)[None, :] < L[:, None]
+    out = np.zeros((B, t_max), dtype=np.float64)
+    out[valid] = advantages(r[valid], v[valid], L, stopped, gamma, lam, r_fail, direct=direct)   # row-major: row after row
+    return out
+
+
 def advantages_f32(rewards, values, lengths, stopped, gamma, lam, r_fail, n_threads=1) -> np.ndarray:
     r = np.ascontiguousarray(rewards, dtype=np.float32)
     v = np.ascontiguousarray(values, dtype=np.float32)

@@ -78,6 +78,7 @@ def lib():
         L.espo_advantages.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp]
         L.espo_advantages_returns.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp]
         L.espo_advantages_stats.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp, vp]
+        L.espo_advantages_padded.argtypes = [vp, vp, vp, vp, i32, i32, f32, f32, f32, vp, vp, vp]
         L.espo_advantages_noalloc.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp]
         L.espo_advantages_reserve.argtypes = [i32, i64]
         L.espo_advantages_status.argtypes = [C.POINTER(C.c_uint32), vp]
@@ -86,7 +87,7 @@ def lib():
         L.espo_last_cuda_error.argtypes = []
         for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_state_view",
                   "espo_compact_active", "espo_state_status", "espo_end_batch", "espo_advantages", "espo_advantages_reserve",
-                  "espo_advantages_status", "espo_advantages_noalloc", "espo_advantages_returns", "espo_advantages_stats",
+                  "espo_advantages_status", "espo_advantages_noalloc", "espo_advantages_returns", "espo_advantages_stats", "espo_advantages_padded",
                   "espo_last_cuda_error"):
             getattr(L, n).restype = C.c_int
         _lib = L
@@ -253,6 +254,28 @@ def espo_advantages_returns(rewards: torch.Tensor, values: torch.Tensor, lengths
                                          total, gamma, lam, r_fail, _dev_ptr(adv_out, "adv_out"),
                                          _dev_ptr(returns_out, "returns_out"), _stream(stream)),
            "espo_advantages_returns")
+
+
+def espo_advantages_padded(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.Tensor, stopped: torch.Tensor,
+                           gamma: float, lam: float, r_fail: float, adv_out: torch.Tensor,
+                           returns_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """TD + GAE (Eq. 4-5, 13) over a padded batch: ``rewards``, ``values`` and the outputs are [B, t_max]; see ``espo.h``."""
+    if rewards.dim() != 2:
+        raise ValueError("rewards must be [B, t_max]")
+    B, t_max = rewards.shape
+    for t, n in ((rewards, "rewards"), (values, "values"), (adv_out, "adv_out")) + \
+            (() if returns_out is None else ((returns_out, "returns_out"),)):
+        if t.dtype != torch.float32 or not t.is_contiguous() or tuple(t.shape) != (B, t_max):
+            raise ValueError(f"{n} must be a contiguous float32 [B, t_max] tensor")
+    if lengths.dtype != torch.int32 or not lengths.is_contiguous() or lengths.numel() != B:
+        raise ValueError("lengths must be a contiguous int32 [B] tensor")
+    if stopped.dtype != torch.uint8 or not stopped.is_contiguous() or stopped.numel() < B:
+        raise ValueError("stopped must be a contiguous uint8 [B] tensor")
+    _check(lib().espo_advantages_padded(_dev_ptr(rewards, "rewards"), _dev_ptr(values, "values"),
+                                        _dev_ptr(lengths, "lengths"), _dev_ptr(stopped, "stopped"), B, t_max,
+                                        gamma, lam, r_fail, _dev_ptr(adv_out, "adv_out"),
+                                        _dev_ptr(returns_out, "returns_out"), _stream(stream)),
+           "espo_advantages_padded")
 
 
 def espo_advantages_stats(rewards: torch.Tensor, values: torch.Tensor, lengths: torch.Tensor, stopped: torch.Tensor,

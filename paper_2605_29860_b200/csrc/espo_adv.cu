@@ -67,6 +67,7 @@ struct AdvArgs {
   float* ret;             // optional: returns A_t + V_t (value targets), same layout as adv; may be null
   double* stats;          // optional: [2] sum of A_t and of A_t^2 over all tokens; may be null
   int B;
+  int t_max;              // > 0: padded layout, trajectory i owns tokens [i*t_max, i*t_max + lengths[i]); 0: packed
   long long total;
   int nchunks;
   double gamma, gl;       // gamma, gamma*lambda
@@ -125,6 +126,26 @@ __global__ void __launch_bounds__(kPrepThreads) espo_adv_prep_kernel(const AdvAr
   if (bad) atomicOr(a.ws.status, ESPO_DEV_BAD_LENGTHS);
 }
 
+// Preparation for the padded layout [B, t_max]: row i starts at token i*t_max, so offsets and chunk owners are
+// plain arithmetic; lengths outside [0, t_max] are reported (the scan clamps them).
+__global__ void __launch_bounds__(kPrepThreads) espo_adv_prep_padded_kernel(const AdvArgs a) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  bool bad = false;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i <= a.B; i += stride) {
+    a.ws.offsets[i] = i * a.t_max;
+    if (i < a.B) {
+      const int len = a.lengths[i];
+      bad |= (len < 0 || len > a.t_max);
+    }
+  }
+  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < a.nchunks; j += stride) {
+    const long long i = j * kAdvChunk / a.t_max;
+    a.ws.chunk_first[j] = (int)(i < a.B ? i : a.B - 1);
+  }
+  if (bad) atomicOr(a.ws.status, ESPO_DEV_BAD_LENGTHS);
+}
+
 // ---------------------------------------------------------------------------------------
 // The scan.
 // ---------------------------------------------------------------------------------------
@@ -155,23 +176,26 @@ __device__ __forceinline__ double shfl_d(double v, int src) { return __shfl_sync
 
 // Shared memory of the scan kernel: a ring of kAdvStages stages, each one chunk of rewards, one chunk of values
 // followed by the value of the token after the chunk, and one flag word per scanning thread (bit e: the thread's
-// token e is the last of a trajectory; bit 16 + e: that trajectory was stopped).
+// token e is the last of a trajectory; bit 16 + e: that trajectory was stopped) and, for the padded layout, one word
+// of padding bits (bit e: the thread's token e belongs to no trajectory).
 constexpr int kAdvVStride = kAdvChunk + 4;      // floats; keeps every stage 16-byte aligned
 constexpr size_t kAdvSmemBytes =
-    (size_t)kAdvStages * (sizeof(float) * kAdvChunk + sizeof(float) * kAdvVStride + sizeof(uint32_t) * kAdvThreads) +
+    (size_t)kAdvStages * (sizeof(float) * kAdvChunk + sizeof(float) * kAdvVStride + 2 * sizeof(uint32_t) * kAdvThreads) +
     2 * kAdvStages * sizeof(uint64_t);
 
 // kAdvThreads threads scan; one more warp (the producer) keeps the ring full and sets the flag words, so that no
 // scanning warp ever waits for a load from global memory.
 // STATS: also the batch sums of A and A^2.  RET: also the returns A_t + V_t; the scanning threads then keep a stage
 // until they have stored, because they read the values from it a second time.
-template <bool STATS, bool RET>
+// PADDED: the arrays are [B, t_max] with padding after every trajectory; padding reads as anything and is written as 0.
+template <bool STATS, bool RET, bool PADDED>
 __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_kernel(const AdvArgs a) {
   extern __shared__ __align__(128) unsigned char adv_smem[];
   float* rbuf = reinterpret_cast<float*>(adv_smem);
   float* vbuf = rbuf + kAdvStages * kAdvChunk;
   uint32_t* fwbuf = reinterpret_cast<uint32_t*>(vbuf + kAdvStages * kAdvVStride);
-  uint64_t* full = reinterpret_cast<uint64_t*>(fwbuf + kAdvStages * kAdvThreads);   // data and flags of the stage are in place
+  uint32_t* pwbuf = fwbuf + kAdvStages * kAdvThreads;
+  uint64_t* full = reinterpret_cast<uint64_t*>(pwbuf + kAdvStages * kAdvThreads);   // data and flags of the stage are in place
   uint64_t* empty = full + kAdvStages;                                                // every scanning thread has read the stage
   __shared__ Map warp_agg[2][kAdvWarps];                    // double-buffered: consecutive chunks alternate
   __shared__ double pw[kAdvPerThread + 1];                   // (gamma*lambda)^i
@@ -205,7 +229,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     double p = 1.0;
     for (int i = 0; i <= kAdvPerThread; ++i) { pw[i] = p; p *= a.gl; }
   }
-  for (int i = tid; i < kAdvStages * kAdvThreads; i += kAdvCtaThreads) fwbuf[i] = 0u;
+  for (int i = tid; i < 2 * kAdvStages * kAdvThreads; i += kAdvCtaThreads) fwbuf[i] = 0u;   // flag and padding words
   __syncthreads();
 
   if (warp == kAdvWarps) {
@@ -257,11 +281,30 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     auto traj_load = [&](int i, int c_hi) -> Traj {
       Traj t{0, 0, 0u};
       if (i <= c_hi) {
-        t.o0 = __ldcg(a.ws.offsets + i);
-        t.o1 = __ldcg(a.ws.offsets + i + 1);
+        if (PADDED) {
+          const int len = a.lengths[i];
+          t.o0 = (long long)i * a.t_max;
+          t.o1 = t.o0 + (len < 0 ? 0 : (len > a.t_max ? a.t_max : len));
+        } else {
+          t.o0 = __ldcg(a.ws.offsets + i);
+          t.o1 = __ldcg(a.ws.offsets + i + 1);
+        }
         t.st = a.stopped[i];
       }
       return t;
+    };
+    // Padded layout: tokens [from, to) belong to no trajectory; every lane calls this with the same arguments and
+    // sets the padding bits of its share of the chunk's words.
+    auto pad_mark = [&](int k, long long from, long long to) {
+      const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+      const long long lo = max(from, max(p0, t_lo)), hi = min(to, min(p0 + kAdvChunk, a.total));
+      if (lo >= hi) return;
+      const int q_lo = (int)(lo - p0), q_hi = (int)(hi - p0);
+      uint32_t* pw = pwbuf + (k % kAdvStages) * kAdvThreads;
+      for (int w = q_lo / kAdvPerThread + lane; w <= (q_hi - 1) / kAdvPerThread; w += 32) {
+        const int b0 = max(q_lo - w * kAdvPerThread, 0), b1 = min(q_hi - w * kAdvPerThread, kAdvPerThread);
+        atomicOr(pw + w, ((1u << (b1 - b0)) - 1u) << b0);
+      }
     };
     auto traj_mark = [&](int k, const Traj& t) {
       const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
@@ -270,6 +313,18 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
       if (t.o1 > t.o0 && t.o1 - 1 >= p_lo && t.o1 - 1 < p_end) {
         const int pos = (int)(t.o1 - 1 - p0);
         atomicOr(fwbuf + (k % kAdvStages) * kAdvThreads + (pos / kAdvPerThread), (1u | (t.st ? 0x10000u : 0u)) << (pos % kAdvPerThread));
+      }
+    };
+
+    // Marks what one round of candidates (lane l holds candidate first + l) contributes to chunk k.
+    auto mark_round = [&](int k, const Traj& t, int first, int c_hi) {
+      traj_mark(k, t);
+      if (PADDED) {
+        const int n = min(32, c_hi - first + 1);
+        for (int j = 0; j < n; ++j) {
+          const long long o0 = __shfl_sync(kFullMask, t.o0, j), o1 = __shfl_sync(kFullMask, t.o1, j);
+          pad_mark(k, o1, o0 + a.t_max);
+        }
       }
     };
 
@@ -286,8 +341,8 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
         if (!mbar_wait_bounded(&empty[stage], (uint32_t)((k / kAdvStages - 1) & 1), nullptr)) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
         if (lane == 0) issue_copies(k);
       }
-      traj_mark(k, t0);
-      for (int i = c_lo + 32 + lane; i <= c_hi; i += 32) traj_mark(k, traj_load(i, c_hi));
+      mark_round(k, t0, c_lo, c_hi);
+      for (int first = c_lo + 32; first <= c_hi; first += 32) mark_round(k, traj_load(first + lane, c_hi), first, c_hi);
       __syncwarp();
       if (lane == 0) mbar_arrive(&full[stage]);             // the flags (and lane 0's ordinary stores) are in place
       c_lo = n_lo; c_hi = n_hi;
@@ -299,7 +354,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
   }
 
   // =============================== scanning warps ===============================
-  unsigned last_mask = 0;
+  unsigned last_mask = 0, pad_mask = 0;
   double d[kAdvPerThread];
   Map m, after;
 
@@ -326,9 +381,15 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     uint32_t* fp = fwbuf + stage * kAdvThreads + tid;
     const uint32_t fw = *fp;
     *fp = 0u;
-    if (!RET) mbar_arrive(&empty[stage]);           // release: this thread's reads and its cleared flag word come first
     last_mask = fw & 0xffffu;
     unsigned fail_mask = fw >> 16;
+    if (PADDED) {
+      uint32_t* pp = pwbuf + stage * kAdvThreads + tid;
+      pad_mask = *pp;
+      *pp = 0u;
+      last_mask |= pad_mask;          // padding cuts the recursion like a trajectory end, with a TD error of 0
+    }
+    if (!RET) mbar_arrive(&empty[stage]);           // release: this thread's reads and its cleared words come first
     {
       // the array's very last token ends a trajectory even if the lengths are inconsistent
       const long long e_last = a.total - 1 - p0 - q0;
@@ -353,7 +414,8 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
         const bool last = (last_mask >> e) & 1u;
         const double vd = (double)v[e];
         const double rd = ((fail_mask >> e) & 1u) ? r_fail_d : (double)r[e];
-        const double de = (last ? rd : fma(a.gamma, vd_next, rd)) - vd;
+        double de = (last ? rd : fma(a.gamma, vd_next, rd)) - vd;
+        if (PADDED) de = ((pad_mask >> e) & 1u) ? 0.0 : de;     // whatever the padding holds never enters
         d[e] = de;
         mb = last ? de : fma(a.gl, mb, de);
         vd_next = vd;
@@ -385,8 +447,15 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     int first = __ldcg(a.ws.chunk_first + (t_hi / kAdvChunk));
     if ((unsigned)first >= (unsigned)a.B) first = a.B;   // only with inconsistent lengths (flagged by the preparation)
     for (int i = first + tid; i < a.B; i += kAdvThreads) {
-      const long long o0 = __ldcg(a.ws.offsets + i);
-      const long long o1 = __ldcg(a.ws.offsets + i + 1);
+      long long o0, o1;
+      if (PADDED) {
+        const int len = a.lengths[i];
+        o0 = (long long)i * a.t_max;
+        o1 = o0 + (len < 0 ? 0 : (len > a.t_max ? a.t_max : len));
+      } else {
+        o0 = __ldcg(a.ws.offsets + i);
+        o1 = __ldcg(a.ws.offsets + i + 1);
+      }
       const int st = a.stopped[i];
       if (o0 > t_hi) break;
       if (o1 > t_hi) { halo_traj = i; halo_end = o1; halo_failed = st; }
@@ -492,8 +561,14 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
 #pragma unroll
         for (int h = 0; h < kAdvPerThread / 4; ++h) {
           const float4 vv = *reinterpret_cast<const float4*>(vs + q0 + 4 * h);
-          __stcs(reinterpret_cast<float4*>(a.ret + p0 + q0) + h,
-                 make_float4(out[4 * h] + vv.x, out[4 * h + 1] + vv.y, out[4 * h + 2] + vv.z, out[4 * h + 3] + vv.w));
+          float4 rt = make_float4(out[4 * h] + vv.x, out[4 * h + 1] + vv.y, out[4 * h + 2] + vv.z, out[4 * h + 3] + vv.w);
+          if (PADDED && pad_mask) {
+            rt.x = ((pad_mask >> (4 * h)) & 1u) ? 0.f : rt.x;
+            rt.y = ((pad_mask >> (4 * h + 1)) & 1u) ? 0.f : rt.y;
+            rt.z = ((pad_mask >> (4 * h + 2)) & 1u) ? 0.f : rt.z;
+            rt.w = ((pad_mask >> (4 * h + 3)) & 1u) ? 0.f : rt.w;
+          }
+          __stcs(reinterpret_cast<float4*>(a.ret + p0 + q0) + h, rt);
         }
       }
     } else {
@@ -501,7 +576,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
       for (int e = 0; e < kAdvPerThread; ++e)
         if (q0 + e >= q_lo && q0 + e < q_hi) {
           a.adv[p0 + q0 + e] = out[e];
-          if (RET) a.ret[p0 + q0 + e] = out[e] + vbuf[(k % kAdvStages) * kAdvVStride + q0 + e];
+          if (RET) a.ret[p0 + q0 + e] = (PADDED && ((pad_mask >> e) & 1u)) ? 0.f : out[e] + vbuf[(k % kAdvStages) * kAdvVStride + q0 + e];
         }
     }
     if (RET) mbar_arrive(&empty[k % kAdvStages]);   // release: the second read of the values comes first
@@ -554,13 +629,15 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
   int dev = 0;
   ESPO_CUDA_TRY(cudaGetDevice(&dev));
   if (dev >= 0 && dev < kMaxDevicesAdv && !attr_set[dev]) {
-    const void* variants[4] = {(const void*)espo_adv_scan_kernel<false, false>, (const void*)espo_adv_scan_kernel<false, true>,
-                               (const void*)espo_adv_scan_kernel<true, false>, (const void*)espo_adv_scan_kernel<true, true>};
+    const void* variants[6] = {(const void*)espo_adv_scan_kernel<false, false, false>, (const void*)espo_adv_scan_kernel<false, true, false>,
+                               (const void*)espo_adv_scan_kernel<true, false, false>, (const void*)espo_adv_scan_kernel<true, true, false>,
+                               (const void*)espo_adv_scan_kernel<false, false, true>, (const void*)espo_adv_scan_kernel<false, true, true>};
     for (const void* f : variants)
       ESPO_CUDA_TRY(cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAdvSmemBytes));
     attr_set[dev] = true;
   }
-  espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
+  if (a.t_max > 0) espo_adv_prep_padded_kernel<<<8, kPrepThreads, 0, s>>>(a);
+  else espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
   ESPO_CUDA_TRY(cudaGetLastError());
   long long grid = (long long)sm_count * kAdvCtasPerSm;
   if (grid > a.nchunks) grid = a.nchunks;
@@ -574,10 +651,12 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (a.stats && a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<true, true>, a));
-  else if (a.stats) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<true, false>, a));
-  else if (a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, true>, a));
-  else ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, false>, a));
+  if (a.t_max > 0 && a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, true, true>, a));
+  else if (a.t_max > 0) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, false, true>, a));
+  else if (a.stats && a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<true, true, false>, a));
+  else if (a.stats) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<true, false, false>, a));
+  else if (a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, true, false>, a));
+  else ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, false, false>, a));
   return ESPO_OK;
 }
 
@@ -680,7 +759,7 @@ int espo_advantages_noalloc(const float* rewards, const float* values, const int
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = nullptr;
   a.stats = nullptr; a.ws.partials = nullptr; a.ws.done = nullptr;
-  a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
+  a.B = B; a.t_max = 0; a.total = total_tokens; a.nchunks = (int)nchunks;
   set_discount(a, gamma, lambda);
   a.r_fail = r_fail;
   a.ws.offsets = (long long*)(b + kNaOffOffsets);
@@ -726,11 +805,41 @@ int espo_advantages_stats(const float* rewards, const float* values, const int32
   AdvArgs a;
   a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = returns_out;
   a.stats = stats_out;
-  a.B = B; a.total = total_tokens; a.nchunks = (int)nchunks;
+  a.B = B; a.t_max = 0; a.total = total_tokens; a.nchunks = (int)nchunks;
   set_discount(a, gamma, lambda);
   a.r_fail = r_fail;
   a.ws = p->ws;
   return launch_advantages(a, p->sm_count, s);
+}
+
+int espo_advantages_padded(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,
+                           int32_t B, int32_t t_max, float gamma, float lambda, float r_fail, float* adv_out,
+                           float* returns_out, void* stream) {
+  using namespace espo;
+  if (B < 0 || t_max < 0) return ESPO_ERR_BAD_SHAPE;
+  if (B == 0 || t_max == 0) return ESPO_OK;
+  if (!rewards || !values || !lengths || !stopped || !adv_out) return ESPO_ERR_NULL;
+  if (((uintptr_t)rewards % 16) || ((uintptr_t)values % 16) || ((uintptr_t)adv_out % 16) || ((uintptr_t)lengths % 4) ||
+      ((uintptr_t)returns_out % 16))
+    return ESPO_ERR_ALIGN;
+  if (gamma != gamma || lambda != lambda || r_fail != r_fail) return ESPO_ERR_BAD_PARAM;
+  const long long total = (long long)B * t_max;
+  const long long nchunks = (total + kAdvChunk - 1) / kAdvChunk;
+  if (nchunks > 0x7fffffffLL) return ESPO_ERR_CAPACITY;
+  int dev;
+  ESPO_CUDA_TRY(cudaGetDevice(&dev));
+  std::lock_guard<std::mutex> lk(g_pool_mu);
+  AdvPool* p;
+  int rc = ensure_pool(dev, B, nchunks, &p);
+  if (rc != ESPO_OK) return rc;
+  AdvArgs a;
+  a.rewards = rewards; a.values = values; a.lengths = lengths; a.stopped = stopped; a.adv = adv_out; a.ret = returns_out;
+  a.stats = nullptr;
+  a.B = B; a.t_max = t_max; a.total = total; a.nchunks = (int)nchunks;
+  set_discount(a, gamma, lambda);
+  a.r_fail = r_fail;
+  a.ws = p->ws;
+  return launch_advantages(a, p->sm_count, (cudaStream_t)stream);
 }
 
 int espo_advantages_returns(const float* rewards, const float* values, const int32_t* lengths, const uint8_t* stopped,

@@ -148,3 +148,38 @@ def test_batch_sums_come_out_of_the_same_pass():
                                torch.empty(0, dtype=torch.uint8, device="cuda"), 1.0, 0.95, -1.0, z, empty)
     torch.cuda.synchronize()
     assert empty.tolist() == [0.0, 0.0]
+
+
+@pytest.mark.parametrize("B,t_max,lo", [(64, 4096, 1), (300, 1000, 0), (1000, 37, 0), (3, 20000, 15000), (1, 5, 5), (5, 1, 0),
+                                        (40, 3072, 3072), (17, 6145, 0)])
+def test_padded_layout(B, t_max, lo):
+    # [B, t_max] batch; the padding holds NaN on the way in and must come back as 0
+    g = torch.Generator("cuda").manual_seed(B * 131 + t_max)
+    L = torch.randint(lo, t_max + 1, (B,), generator=g, device="cuda", dtype=torch.int64).to(torch.int32)
+    s = (torch.rand(B, generator=g, device="cuda") < 0.4).to(torch.uint8)
+    r = torch.randn(B, t_max, generator=g, device="cuda") * 0.5
+    v = torch.randn(B, t_max, generator=g, device="cuda") * 0.5
+    pad = torch.arange(t_max, device="cuda")[None, :] >= L[:, None]
+    r[pad] = float("nan"); v[pad] = float("nan")
+    for gamma, lam in ((1.0, 1.0), (0.99, 0.95)):
+        adv = torch.full((B, t_max), 7.0, device="cuda"); ret = torch.full((B, t_max), 7.0, device="cuda")
+        espo.espo_advantages_padded(r, v, L, s, gamma, lam, -1.0, adv, ret)
+        adv2 = torch.full((B, t_max), 7.0, device="cuda")
+        espo.espo_advantages_padded(r, v, L, s, gamma, lam, -1.0, adv2)
+        torch.cuda.synchronize()
+        assert espo.espo_advantages_status() == 0
+        ref = oracle.advantages_padded(r.cpu().numpy(), v.cpu().numpy(), L.cpu().numpy(), s.cpu().numpy(),
+                                       float(np.float32(gamma)), float(np.float32(lam)), -1.0)
+        got = adv.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref) <= 1e-5 + 1e-4 * np.abs(ref))
+        assert torch.equal(adv, adv2)
+        assert np.all(got[pad.cpu().numpy()] == 0.0)
+        want_ret = ref + np.where(pad.cpu().numpy(), 0.0, np.nan_to_num(v.cpu().numpy().astype(np.float64)))
+        got_ret = ret.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got_ret - want_ret) <= 2e-5 + 1e-4 * np.abs(want_ret))
+        assert np.all(got_ret[pad.cpu().numpy()] == 0.0)
+    # a length outside [0, t_max] is reported, not trapped
+    bad = L.clone(); bad[0] = t_max + 3
+    espo.espo_advantages_padded(torch.nan_to_num(r), torch.nan_to_num(v), bad, s, 1.0, 0.95, -1.0, adv)
+    torch.cuda.synchronize()
+    assert espo.espo_advantages_status() & espo.ESPO_DEV_BAD_LENGTHS

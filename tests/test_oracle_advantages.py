@@ -118,3 +118,27 @@ def test_float32_threaded_entry_point_agrees():
     a = oracle.advantages(r32.astype(np.float64), v32.astype(np.float64), L, s, 1.0, 0.95, -1.0)
     b = oracle.advantages_f32(r32, v32, L, s, 1.0, 0.95, -1.0, n_threads=4)
     np.testing.assert_array_equal(a, b)
+
+
+def test_padded_layout_is_the_literal_sum_row_by_row():
+    # Eq. 5 written out for every row of a [B, t_max] batch on its own, padding filled with NaN
+    rng = np.random.default_rng(5)
+    B, t_max, gamma, lam, r_fail = 7, 23, 0.97, 0.9, -1.0
+    L = np.array([0, 1, 23, 5, 22, 2, 11], dtype=np.int32)
+    stopped = np.array([1, 1, 0, 1, 0, 0, 1], dtype=np.uint8)
+    r = rng.normal(0, 0.5, size=(B, t_max)); v = rng.normal(0, 0.5, size=(B, t_max))
+    pad = np.arange(t_max)[None, :] >= L[:, None]
+    r[pad] = np.nan; v[pad] = np.nan
+    got = oracle.advantages_padded(r, v, L, stopped, gamma, lam, r_fail)
+    want = np.zeros((B, t_max))
+    for i in range(B):
+        n = int(L[i])
+        rr = r[i, :n].copy()
+        if n and stopped[i]:
+            rr[n - 1] = r_fail                                   # Eq. 13 replaces the last reward
+        vv = np.append(v[i, :n], 0.0)                            # nothing is bootstrapped past the last token
+        delta = rr + gamma * vv[1:] - vv[:-1]                    # Eq. 4
+        for t in range(n):
+            want[i, t] = sum((gamma * lam) ** l * delta[t + l] for l in range(n - t))   # Eq. 5
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    assert np.all(got[pad] == 0.0)
