@@ -196,6 +196,47 @@ int espo_end_batch(espo_state* st, float alpha_ema, float eta_beta, float tau, f
                    float beta_max, int32_t first_update, espo_params* params_inout,
                    double* stats_out, void* stream);
 
+/* ---- vocabulary shards (a tensor-parallel LM head leaves every GPU with V/N of each logit row) ----
+ * The paper samples from whole rows (Algorithm 1); this pair of calls computes the same step when a row's logits
+ * are spread over several buffers.  Every shard reduces its part of the rows to one espo_partial per row
+ * (espo_step_partial), the partials of all shards are brought together (one all-gather of 32 bytes per row and
+ * shard when the shards live on different GPUs; the library does not communicate) and espo_step_merge finishes the
+ * step on the trajectory state: regret, normalisation, smoothing, stop rule, bookkeeping (Eq. 6, 9-11), exactly as
+ * espo_step does.  Only the flat sampler is offered: its Gumbel draws belong to token ids, so the perturbed maximum
+ * over the shards is the perturbed maximum over the row and the token does not depend on how the row is cut. */
+typedef struct espo_partial {
+  float m;             /* largest logit of the shard's part of the row (-inf if it has no finite entry)           */
+  float s;             /* sum over the part of exp((x - m) / temperature)                                          */
+  float best;          /* largest perturbed score x/T + G of the part (greedy: the largest logit)                  */
+  int32_t best_id;     /* global token id that attains it, lowest id on ties; -1: none                             */
+  float x_best;        /* that token's logit                                                                        */
+  uint32_t flags;      /* bit 0: the part held NaN or +inf; bit 1: nothing computed (bad slot or ended trajectory) */
+  uint32_t reserved[2];
+} espo_partial;        /* 32 bytes */
+
+/* One shard's share of a decode step.  Reads the state (step counter and slot choose the random stream) and writes
+ * partial_out; changes nothing else, so the shards of a step may run in any order or on different GPUs with
+ * replicas of the state.
+ *   logits_shard   device [n_rows, v_shard] with row_stride elements between rows, dtype as for espo_step
+ *   vocab_offset   global id of the shard's first logit; a multiple of 4; vocab_offset + v_shard <= V
+ *   partial_out    device espo_partial [n_rows], 16-byte aligned
+ *   params         sampler must be ESPO_SAMPLER_FLAT (else ESPO_ERR_BAD_PARAM); temperature 0 = greedy
+ * Calls that use the same state must not overlap on the device (they share its scratch).
+ * Errors: NULL, BAD_SHAPE, BAD_DTYPE, BAD_PARAM, ALIGN, CAPACITY, CUDA. */
+int espo_step_partial(const void* logits_shard, int32_t logits_dtype, int64_t row_stride, int32_t v_shard,
+                      int32_t vocab_offset, const int32_t* row_ids, int32_t n_rows, espo_state* st,
+                      const espo_params* params, espo_partial* partial_out, void* stream);
+
+/* Merges the shards' partials and commits the step, with the outputs and state changes of espo_step.
+ *   partials      device espo_partial: shard k's result for row r at partials[k * shard_stride + r]
+ *   n_shards >= 1, shard_stride >= n_rows (elements)
+ *   values, row_ids, tokens_out, stop_out, params: as for espo_step, with the same params as the partial calls
+ * A row is marked ESPO_ROW_BAD if any shard flagged NaN / +inf or no shard held a finite logit.
+ * Errors: NULL, BAD_SHAPE, BAD_DTYPE, BAD_PARAM, ALIGN, CAPACITY, CUDA. */
+int espo_step_merge(const espo_partial* partials, int32_t n_shards, int64_t shard_stride, const void* values,
+                    int32_t values_dtype, const int32_t* row_ids, int32_t n_rows, espo_state* st,
+                    const espo_params* params, int32_t* tokens_out, uint8_t* stop_out, void* stream);
+
 /* Copy the sticky device status word (ESPO_DEV_* bits) to *host_out.  Synchronises `stream`. */
 int espo_state_status(espo_state* st, uint32_t* host_out, void* stream);
 

@@ -71,6 +71,8 @@ def lib():
         L.espo_free_state.restype = None
         L.espo_set_launch_config.argtypes = [vp, i32, i32, i32]
         L.espo_step.argtypes = [vp, i32, i64, vp, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp, vp]
+        L.espo_step_partial.argtypes = [vp, i32, i64, i32, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp]
+        L.espo_step_merge.argtypes = [vp, i32, i64, vp, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp, vp]
         L.espo_state_view.argtypes = [vp] + [C.POINTER(vp)] * 11
         L.espo_compact_active.argtypes = [vp, vp, vp, vp]
         L.espo_state_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
@@ -85,7 +87,8 @@ def lib():
         L.espo_strerror.argtypes = [C.c_int]
         L.espo_strerror.restype = C.c_char_p
         L.espo_last_cuda_error.argtypes = []
-        for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_state_view",
+        for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_step_partial",
+                  "espo_step_merge", "espo_state_view",
                   "espo_compact_active", "espo_state_status", "espo_end_batch", "espo_advantages", "espo_advantages_reserve",
                   "espo_advantages_status", "espo_advantages_noalloc", "espo_advantages_returns", "espo_advantages_stats", "espo_advantages_padded",
                   "espo_last_cuda_error"):
@@ -184,6 +187,51 @@ def espo_step(logits: torch.Tensor, values: torch.Tensor, state: EspoState, para
                            _dev_ptr(row_ids, "row_ids"), n, state.handle, C.byref(params),
                            _dev_ptr(tokens_out, "tokens_out"), _dev_ptr(stop_out, "stop_out"), _stream(stream)),
            "espo_step")
+
+
+PARTIAL_FLOATS = 8   # an espo_partial is 32 bytes; tensors of partials are float32 [..., 8] (ids and flags bit-cast)
+
+
+def espo_step_partial(logits_shard: torch.Tensor, vocab_offset: int, state: EspoState, params: espo_params,
+                      partial_out: torch.Tensor, row_ids: Optional[torch.Tensor] = None, n_rows: Optional[int] = None,
+                      stream=None) -> None:
+    """One vocabulary shard's share of a decode step: ``logits_shard`` is [n_rows, v_shard], its first column is
+    token ``vocab_offset``; writes one espo_partial per row into ``partial_out`` (float32 [n_rows, 8]); see ``espo.h``."""
+    if logits_shard.dim() != 2 or logits_shard.stride(1) != 1:
+        raise ValueError("logits_shard must be [n_rows, v_shard] with unit stride along the vocabulary")
+    n = logits_shard.shape[0] if n_rows is None else n_rows
+    if partial_out.dtype != torch.float32 or not partial_out.is_contiguous() or partial_out.numel() < n * PARTIAL_FLOATS:
+        raise ValueError("partial_out must be a contiguous float32 tensor of n_rows * 8 elements")
+    if row_ids is not None and (row_ids.dtype != torch.int32 or row_ids.numel() < n):
+        raise ValueError("row_ids must be int32 [n_rows]")
+    _check(lib().espo_step_partial(_dev_ptr(logits_shard, "logits_shard"), _dtype_code(logits_shard, "logits_shard"),
+                                   logits_shard.stride(0), logits_shard.shape[1], vocab_offset,
+                                   _dev_ptr(row_ids, "row_ids"), n, state.handle, C.byref(params),
+                                   _dev_ptr(partial_out, "partial_out"), _stream(stream)),
+           "espo_step_partial")
+
+
+def espo_step_merge(partials: torch.Tensor, values: torch.Tensor, state: EspoState, params: espo_params,
+                    tokens_out: torch.Tensor, stop_out: torch.Tensor, row_ids: Optional[torch.Tensor] = None,
+                    n_rows: Optional[int] = None, stream=None) -> None:
+    """Merges the shards' partials (float32 [n_shards, rows, 8]) and commits the step like ``espo_step``; see ``espo.h``."""
+    if partials.dim() != 3 or partials.shape[2] != PARTIAL_FLOATS or partials.dtype != torch.float32 or \
+            not partials.is_contiguous():
+        raise ValueError("partials must be a contiguous float32 [n_shards, rows, 8] tensor")
+    n = partials.shape[1] if n_rows is None else n_rows
+    if tokens_out.dtype != torch.int32 or stop_out.dtype != torch.uint8:
+        raise ValueError("tokens_out must be int32 and stop_out uint8")
+    if row_ids is not None and row_ids.dtype != torch.int32:
+        raise ValueError("row_ids must be int32")
+    if not values.is_contiguous() or not tokens_out.is_contiguous() or not stop_out.is_contiguous():
+        raise ValueError("values, tokens_out and stop_out must be contiguous")
+    if min(values.numel(), tokens_out.numel(), stop_out.numel()) < n or (row_ids is not None and row_ids.numel() < n):
+        raise ValueError("an argument is shorter than n_rows")
+    _check(lib().espo_step_merge(_dev_ptr(partials, "partials"), partials.shape[0], partials.shape[1],
+                                 _dev_ptr(values, "values"), _dtype_code(values, "values"), _dev_ptr(row_ids, "row_ids"),
+                                 n, state.handle, C.byref(params), _dev_ptr(tokens_out, "tokens_out"),
+                                 _dev_ptr(stop_out, "stop_out"), _stream(stream)),
+           "espo_step_merge")
 
 
 class _DevArray:

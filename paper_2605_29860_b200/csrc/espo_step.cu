@@ -81,6 +81,12 @@ struct StepArgs {
   // outputs
   int32_t* tokens_out;
   uint8_t* stop_out;
+  // vocabulary shards (espo_step_partial / espo_step_merge)
+  int vocab_offset;              // global id of the shard's first logit (0 for a whole row)
+  espo_partial* partial_out;     // not null: write the row's partial result here instead of updating the state
+  const espo_partial* partials;  // merge: [n_shards][shard_stride] partial results
+  int n_shards;
+  long long shard_stride;
 };
 
 struct StepCtrl {
@@ -220,7 +226,7 @@ __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned c
     int best_id = -1;
 #pragma unroll
     for (int q = 0; q < 32 / 4; ++q) {
-      const int first = block * kBlockIds + id_in_block<ES>(4 * q, lane);
+      const int first = a.vocab_offset + block * kBlockIds + id_in_block<ES>(4 * q, lane);   // global id, a multiple of 4
       const uint4 rnd = philox4x32_10((uint32_t)first >> 2, ds.step, ds.slot, ds.batch_bits | 0u, ds.k0, ds.k1);
       const uint32_t wd[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
@@ -280,7 +286,8 @@ __device__ __forceinline__ RowPre prefetch_row(const StepArgs& a, int row) {
     p.sum_g = a.sum_g[p.slot];
     p.sum_g2 = a.sum_g2[p.slot];
   }
-  if (a.values_bf16) p.v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(a.values) + row) << 16);
+  if (!a.values) p.v = 0.f;
+  else if (a.values_bf16) p.v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(a.values) + row) << 16);
   else p.v = __ldg(reinterpret_cast<const float*>(a.values) + row);
   return p;
 }
@@ -299,6 +306,64 @@ __device__ __forceinline__ float sum_exp2_32(const float (&x)[kSubIds], float m,
   return (acc0.x + acc0.y) + (acc1.x + acc1.y);
 }
 
+// What one thread does once a row's token is known: regret, normalisation, smoothing, stop rule and bookkeeping
+// (Eq. 6, 9, 10, 11; Algorithm 1).  M: largest logit; log_S = ln sum_a exp((x_a - M)/T); l_tok: the token's logit;
+// S, run_u: the sums the entropy needs (relative to M).
+__device__ __forceinline__ void commit_row(const StepArgs& a, int row, const RowPre& pre, const DrawStream& ds, float M,
+                                           float S, float log_S, float run_u, float l_tok, int token, bool no_ticket) {
+  const int slot = pre.slot;
+  const int t_now = pre.t_now;
+  {
+    // Eq. 6: the normaliser cancels; Eq. 9; Eq. 10; Eq. 11.
+    const float g = a.greedy ? 0.f : (M - l_tok) * a.inv_temp;
+    const float logp = a.greedy ? 0.f : (-g - log_S);
+    float gt = (g - a.mu_g) * a.inv_sigma;
+    gt = fminf(fmaxf(gt, -a.clip_c), a.clip_c);
+    const float z = fmaf(a.alpha_s, pre.z_prev, a.one_minus_alpha * gt);
+    const float v = pre.v;
+    const bool v_nan = (v != v);
+    if (v_nan) atomicOr(a.dev_status, ESPO_DEV_NAN_VALUE);
+    const float thr = a.beta * fmaxf(v, a.eps);
+    bool rule;
+    if (a.stop_mode == ESPO_STOP_ESPO) rule = !v_nan && (z > thr);                 // Eq. 11
+    else if (a.stop_mode == ESPO_STOP_VALUE_ONLY) rule = !v_nan && (v < a.tau);
+    else if (a.stop_mode == ESPO_STOP_REGRET_ONLY) rule = (z > a.tau);
+    else rule = (uniform_at(ds, 3u, 0u) < a.p_random);
+    const bool fires = a.warmup_complete && rule;
+
+    a.z[slot] = z;
+    a.g[slot] = g;
+    a.g_tilde[slot] = gt;
+    a.logp[slot] = logp;
+    a.sum_g[slot] = pre.sum_g + (double)g;
+    a.sum_g2[slot] = pre.sum_g2 + (double)g * (double)g;
+    if (a.want_entropy) {
+      // H = ln S - ln2 * U / S with S, U the sums of e and of e*t relative to the row maximum
+      const float h = a.greedy ? 0.f : fmaxf(log_S - 0.6931471805599453f * run_u / S, 0.f);
+      a.entropy[slot] = h;
+      a.sum_h[slot] += (double)h;
+    }
+    const int t_new = t_now + 1;
+    a.t[slot] = t_new;
+    uint8_t stop = 0;
+    if (a.eos_token >= 0 && token == a.eos_token) {
+      a.status[slot] = ESPO_ROW_EOS;
+    } else if (fires && a.shadow) {
+      if (a.t_stop[slot] < 0) a.t_stop[slot] = t_now;        // remembered, not acted upon
+      if (t_new >= a.t_max) a.status[slot] = ESPO_ROW_TMAX;
+    } else if (fires) {
+      a.status[slot] = ESPO_ROW_STOPPED;
+      a.t_stop[slot] = t_now;
+      stop = 1;
+    } else if (t_new >= a.t_max) {
+      a.status[slot] = ESPO_ROW_TMAX;
+    }
+    a.tokens_out[row] = token;
+    a.stop_out[row] = stop;
+    if (!no_ticket) a.ticket[row] = 0;   // ready for the next launch
+  }
+}
+
 // All perturbed scores below are "x/T + G" on the absolute scale of the logits, with the
 // Gumbel written through its exponential draw E = -ln u:  G = -ln E, and for a group with
 // log-sum-exp  m/T + ln s  the score is  m/T + ln(s / E).
@@ -306,9 +371,24 @@ template <int ES, int SAMPLER>
 __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, const RowPre pre, const void* rec_row,
                                           bool rec_local, bool no_ticket, const float* noise) {
   const float NINF = __int_as_float(0xff800000);
+  // only the flat sampler's kernels serve vocabulary shards
+  const bool partial = (SAMPLER == ESPO_SAMPLER_FLAT) && a.partial_out != nullptr;
   const int slot = pre.slot;
-  if (slot < 0) { mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, no_ticket); return; }
-  if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, slot, lane, -1, 0u, -1, no_ticket); return; }   // finished: untouched
+  // A vocabulary shard reports instead of acting: `flags` tells the merge what happened (bit 0: the shard's part of
+  // the row held NaN or +inf; bit 1: nothing was computed because the slot is bad or the trajectory has ended).
+  auto report = [&](unsigned flags) {
+    if (lane == 0) {
+      espo_partial pr;
+      pr.m = NINF; pr.s = 0.f; pr.best = NINF; pr.best_id = -1; pr.x_best = NINF; pr.flags = flags; pr.reserved[0] = 0u; pr.reserved[1] = 0u;
+      a.partial_out[row] = pr;
+      if (!no_ticket) a.ticket[row] = 0;
+    }
+  };
+  if (slot < 0) { if (partial) report(2u); else mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, no_ticket); return; }
+  if (pre.status != ESPO_ROW_ACTIVE) {   // finished: untouched
+    if (partial) report(2u); else mark_row(a, row, slot, lane, -1, 0u, -1, no_ticket);
+    return;
+  }
   const int t_now = pre.t_now;
   const unsigned char* row_base = a.logits + (size_t)row * a.row_stride_bytes;
   const DrawStream ds{a.key0, a.key1, (uint32_t)t_now, (uint32_t)slot, a.batch_bits};
@@ -415,10 +495,15 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
   }
   const float M = run_m, S = run_s;
   const float log_S = logf(S);   // needed at the very end; started before the loads below
-  poisoned = __any_sync(kFullMask, poisoned) || !(M > NINF) || isinf(M);
-  if (poisoned) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, no_ticket); return; }
+  // (a shard may hold no finite logit at all; a whole row may not)
+  poisoned = __any_sync(kFullMask, poisoned) || M == __int_as_float(0x7f800000) || M != M;
+  poisoned = poisoned || (!partial && (!(M > NINF) || isinf(M)));
+  if (poisoned) { if (partial) report(1u); else mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, no_ticket); return; }
   warp_argmax(best, best_i);
-  if (best_i < 0) { mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, no_ticket); return; }   // nothing to pick from
+  if (best_i < 0) {   // nothing to pick from
+    if (partial) report(0u); else mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, no_ticket);
+    return;
+  }
 
   int token;
   float l_tok;
@@ -487,59 +572,22 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       l_tok = __shfl_sync(kFullMask, mine, token & 31);
     }
   } else {
-    token = best_i;
-    l_tok = load_logit<ES>(row_base, token);
+    token = best_i;                                             // a global id
+    l_tok = load_logit<ES>(row_base, token - a.vocab_offset);
   }
+  if (a.greedy || SAMPLER == ESPO_SAMPLER_HIER) token += a.vocab_offset;
 
-  if (lane == 0) {
-    // Eq. 6: the normaliser cancels; Eq. 9; Eq. 10; Eq. 11.
-    const float g = a.greedy ? 0.f : (M - l_tok) * a.inv_temp;
-    const float logp = a.greedy ? 0.f : (-g - log_S);
-    float gt = (g - a.mu_g) * a.inv_sigma;
-    gt = fminf(fmaxf(gt, -a.clip_c), a.clip_c);
-    const float z = fmaf(a.alpha_s, pre.z_prev, a.one_minus_alpha * gt);
-    const float v = pre.v;
-    const bool v_nan = (v != v);
-    if (v_nan) atomicOr(a.dev_status, ESPO_DEV_NAN_VALUE);
-    const float thr = a.beta * fmaxf(v, a.eps);
-    bool rule;
-    if (a.stop_mode == ESPO_STOP_ESPO) rule = !v_nan && (z > thr);                 // Eq. 11
-    else if (a.stop_mode == ESPO_STOP_VALUE_ONLY) rule = !v_nan && (v < a.tau);
-    else if (a.stop_mode == ESPO_STOP_REGRET_ONLY) rule = (z > a.tau);
-    else rule = (uniform_at(ds, 3u, 0u) < a.p_random);
-    const bool fires = a.warmup_complete && rule;
-
-    a.z[slot] = z;
-    a.g[slot] = g;
-    a.g_tilde[slot] = gt;
-    a.logp[slot] = logp;
-    a.sum_g[slot] = pre.sum_g + (double)g;
-    a.sum_g2[slot] = pre.sum_g2 + (double)g * (double)g;
-    if (a.want_entropy) {
-      // H = ln S - ln2 * U / S with S, U the sums of e and of e*t relative to the row maximum
-      const float h = a.greedy ? 0.f : fmaxf(log_S - 0.6931471805599453f * run_u / S, 0.f);
-      a.entropy[slot] = h;
-      a.sum_h[slot] += (double)h;
+  if (partial) {
+    // a vocabulary shard: leave what the merge needs and do not touch the state
+    if (lane == 0) {
+      espo_partial pr;
+      pr.m = M; pr.s = S; pr.best = best; pr.best_id = token; pr.x_best = l_tok; pr.flags = 0u; pr.reserved[0] = 0u; pr.reserved[1] = 0u;
+      a.partial_out[row] = pr;
+      if (!no_ticket) a.ticket[row] = 0;   // ready for the next launch
     }
-    const int t_new = t_now + 1;
-    a.t[slot] = t_new;
-    uint8_t stop = 0;
-    if (a.eos_token >= 0 && token == a.eos_token) {
-      a.status[slot] = ESPO_ROW_EOS;
-    } else if (fires && a.shadow) {
-      if (a.t_stop[slot] < 0) a.t_stop[slot] = t_now;        // remembered, not acted upon
-      if (t_new >= a.t_max) a.status[slot] = ESPO_ROW_TMAX;
-    } else if (fires) {
-      a.status[slot] = ESPO_ROW_STOPPED;
-      a.t_stop[slot] = t_now;
-      stop = 1;
-    } else if (t_new >= a.t_max) {
-      a.status[slot] = ESPO_ROW_TMAX;
-    }
-    a.tokens_out[row] = token;
-    a.stop_out[row] = stop;
-    if (!no_ticket) a.ticket[row] = 0;   // ready for the next launch
+    return;
   }
+  if (lane == 0) commit_row(a, row, pre, ds, M, S, log_S, run_u, l_tok, token, no_ticket);
 }
 
 // -------------------------------------------------------------------------------------------
@@ -873,6 +921,40 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_kernel(const __g
   drain_queue<ES, SAMPLER>(a, cr, ctrl, tb, lane);
 }
 
+// -------------------------------------------------------------------------------------------
+// Vocabulary shards: one thread per row merges the shards' partial results and commits the row.
+// -------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(64) espo_merge_kernel(const __grid_constant__ StepArgs a) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= a.n_rows) return;
+  const float NINF = __int_as_float(0xff800000);
+  const RowPre pre = prefetch_row(a, row);
+  if (pre.slot < 0) { mark_row(a, row, 0, 0, -1, ESPO_DEV_BAD_SLOT, -1, true); return; }
+  if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, pre.slot, 0, -1, 0u, -1, true); return; }   // finished: untouched
+  // one pass over the shards: running maximum with the sum rescaled whenever the maximum moves
+  float M = NINF, S = 0.f, best = NINF, x_best = NINF;
+  int best_id = -1;
+  bool poisoned = false;
+#pragma unroll 4
+  for (int k = 0; k < a.n_shards; ++k) {
+    const espo_partial pr = a.partials[(long long)k * a.shard_stride + row];
+    poisoned |= (pr.flags & 1u) != 0u || !(pr.s >= 0.f) || isinf(pr.s);
+    if (pr.s > 0.f) {
+      const float Mn = fmaxf(M, pr.m);
+      S = S * ex2_approx((M - Mn) * a.k2) + pr.s * ex2_approx((pr.m - Mn) * a.k2);   // M = -inf: S is 0 and stays 0
+      M = Mn;
+    }
+    if (pr.best_id >= 0 && (best_id < 0 || pr.best > best || (pr.best == best && pr.best_id < best_id))) {
+      best = pr.best; best_id = pr.best_id; x_best = pr.x_best;      // equal scores: the lowest id wins
+    }
+  }
+  poisoned |= !(M > NINF) || isinf(M);
+  if (poisoned) { mark_row(a, row, pre.slot, 0, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true); return; }
+  if (best_id < 0) { mark_row(a, row, pre.slot, 0, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true); return; }
+  const DrawStream ds{a.key0, a.key1, (uint32_t)pre.t_now, (uint32_t)pre.slot, a.batch_bits};
+  commit_row(a, row, pre, ds, M, S, logf(S), 0.f, x_best, best_id, true);
+}
+
 }  // namespace espo
 
 // ===========================================================================================
@@ -1081,15 +1163,9 @@ int espo_set_launch_config(espo_state* st, int32_t consumer_warps, int32_t stage
   return ESPO_OK;
 }
 
-int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, const void* values, int32_t values_dtype,
-              const int32_t* row_ids, int32_t n_rows, espo_state* st, const espo_params* p, int32_t* tokens_out,
-              uint8_t* stop_out, void* stream) {
+// Checks the frozen parameters and digests them into the kernel's arguments (everything but shapes and pointers).
+static int fill_params(espo::StepArgs& a, const espo_state* st, const espo_params* p) {
   using namespace espo;
-  if (!st || !p) return ESPO_ERR_NULL;
-  if (n_rows < 0) return ESPO_ERR_BAD_SHAPE;
-  if (n_rows > st->capacity) return ESPO_ERR_CAPACITY;
-  if ((logits_dtype != ESPO_F32 && logits_dtype != ESPO_BF16) || (values_dtype != ESPO_F32 && values_dtype != ESPO_BF16))
-    return ESPO_ERR_BAD_DTYPE;
   if (!(p->temperature >= 0.f) || isinf(p->temperature)) return ESPO_ERR_BAD_PARAM;
   if (!(p->sigma2_g >= 0.f) || !(p->sigma2_g + p->delta > 0.f) || !(p->clip_c > 0.f)) return ESPO_ERR_BAD_PARAM;
   if (!(p->alpha_s >= 0.f && p->alpha_s < 1.f) || p->t_max < 1) return ESPO_ERR_BAD_PARAM;
@@ -1099,31 +1175,73 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
       !(p->p_random >= 0.f && p->p_random <= 1.f))
     return ESPO_ERR_BAD_PARAM;
   if (p->want_entropy && p->sampler != ESPO_SAMPLER_HIER) return ESPO_ERR_BAD_PARAM;   // the flat sampler's records are full
+  a.capacity = st->capacity;
+  a.z = st->z; a.g = st->g; a.g_tilde = st->g_tilde; a.logp = st->logp;
+  a.t = st->t; a.t_stop = st->t_stop; a.status = st->status; a.sum_g = st->sum_g; a.sum_g2 = st->sum_g2; a.entropy = st->entropy; a.sum_h = st->sum_h;
+  a.records = st->records; a.ticket = st->ticket; a.dev_status = st->dev_status;
+  a.greedy = (p->temperature == 0.f);
+  const double inv_t = a.greedy ? 1.0 : 1.0 / (double)p->temperature;
+  a.inv_temp = (float)inv_t;
+  a.k2 = (float)(inv_t * 1.4426950408889634074);
+  a.mu_g = p->mu_g;
+  a.inv_sigma = (float)(1.0 / sqrt((double)p->sigma2_g + (double)p->delta));
+  a.clip_c = p->clip_c;
+  a.alpha_s = p->alpha_s;
+  a.one_minus_alpha = 1.0f - p->alpha_s;
+  a.beta = p->beta; a.eps = p->eps;
+  a.warmup_complete = p->warmup_complete; a.t_max = p->t_max; a.eos_token = p->eos_token;
+  a.want_entropy = p->want_entropy != 0;
+  a.stop_mode = p->stop_mode; a.shadow = p->shadow != 0; a.tau = p->tau; a.p_random = p->p_random;
+  a.key0 = (uint32_t)(st->seed & 0xffffffffull);
+  a.key1 = (uint32_t)(st->seed >> 32);
+  a.batch_bits = (uint32_t)(st->batch_id << 2);
+  return ESPO_OK;
+}
+
+// One launch of the step kernel over rows of `v_eff` logits whose first id is `vocab_offset`: the whole vocabulary
+// (espo_step) or one shard of it (espo_step_partial, which passes `partial_out`).
+static int step_launch(const void* logits, int32_t logits_dtype, int64_t row_stride, const void* values, int32_t values_dtype,
+                       const int32_t* row_ids, int32_t n_rows, espo_state* st, const espo_params* p, int32_t* tokens_out,
+                       uint8_t* stop_out, int32_t v_eff, int32_t vocab_offset, espo_partial* partial_out, void* stream) {
+  using namespace espo;
+  if (!st || !p) return ESPO_ERR_NULL;
+  if (n_rows < 0) return ESPO_ERR_BAD_SHAPE;
+  if (n_rows > st->capacity) return ESPO_ERR_CAPACITY;
+  if ((logits_dtype != ESPO_F32 && logits_dtype != ESPO_BF16) || (values_dtype != ESPO_F32 && values_dtype != ESPO_BF16))
+    return ESPO_ERR_BAD_DTYPE;
+  StepArgs a;
+  memset(&a, 0, sizeof(a));
+  {
+    const int rc = fill_params(a, st, p);
+    if (rc != ESPO_OK) return rc;
+  }
   if (n_rows == 0) return ESPO_OK;
-  if (!logits || !values || !tokens_out || !stop_out) return ESPO_ERR_NULL;
-  if (row_stride < st->V) return ESPO_ERR_BAD_SHAPE;
+  if (!logits) return ESPO_ERR_NULL;
+  if (!partial_out && (!values || !tokens_out || !stop_out)) return ESPO_ERR_NULL;
+  if (row_stride < v_eff) return ESPO_ERR_BAD_SHAPE;
+  const int nblk_eff = (v_eff + kBlockIds - 1) / kBlockIds;
   const int es = (logits_dtype == ESPO_BF16) ? 2 : 4;
   const int ves = (values_dtype == ESPO_BF16) ? 2 : 4;
   if (((uintptr_t)logits % es) || ((uintptr_t)values % ves) || ((uintptr_t)tokens_out % 4) ||
-      (row_ids && ((uintptr_t)row_ids % 4)))
+      (row_ids && ((uintptr_t)row_ids % 4)) || ((uintptr_t)partial_out % 16))
     return ESPO_ERR_ALIGN;
 
-  StepArgs a;
-  memset(&a, 0, sizeof(a));
+  a.vocab_offset = vocab_offset;
+  a.partial_out = partial_out;
   a.logits = static_cast<const unsigned char*>(logits);
   a.row_stride_bytes = row_stride * es;
   a.values = values;
   a.values_bf16 = (values_dtype == ESPO_BF16);
   a.row_ids = row_ids;
-  a.n_rows = n_rows; a.V = st->V; a.capacity = st->capacity;
-  a.nblk = st->nblk;
-  a.total_blocks = (long long)n_rows * st->nblk;
+  a.n_rows = n_rows; a.V = v_eff;
+  a.nblk = nblk_eff;
+  a.total_blocks = (long long)n_rows * nblk_eff;
   a.stage_bytes = kBlockIds * es;
   // Launch shape: ctas_per_sm CTAs of `warps` streaming warps (+1 finalizer warp), `stages` blocks in flight per warp.
   int ctas_per_sm = st->cfg_ctas_per_sm ? st->cfg_ctas_per_sm : 1;
   // Finalizer warps per CTA: one row takes a warp about 5 us to finalize, and an SM streams a row in
   // row_bytes / ~43 GB/s; short rows need several finalizers to keep up with the streaming warps.
-  const double row_us = (double)st->V * es / 43e3;
+  const double row_us = (double)v_eff * es / 43e3;
   int fin = (int)ceil(5.0 / (row_us * ctas_per_sm));
   fin = fin < 1 ? 1 : (fin > 8 ? 8 : fin);
   const int max_warps = (kMaxStepThreads / 32 < 64 / ctas_per_sm) ? kMaxStepThreads / 32 : 64 / ctas_per_sm;
@@ -1157,36 +1275,66 @@ int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, cons
   if (per_warp < stages) stages = (int)per_warp;
   a.warps = warps;
   a.fin_warps = fin;
-  a.run_len = (st->nblk >= 64) ? 1 : (st->nblk >= 32 ? 4 : (st->nblk >= 8 ? 2 : 1));
+  a.run_len = (nblk_eff >= 64) ? 1 : (nblk_eff >= 32 ? 4 : (nblk_eff >= 8 ? 2 : 1));
   a.stages = stages;
   const size_t smem = footprint(warps, stages);
   if (smem > (size_t)st->max_smem) return ESPO_ERR_CAPACITY;
 
-  a.z = st->z; a.g = st->g; a.g_tilde = st->g_tilde; a.logp = st->logp;
-  a.t = st->t; a.t_stop = st->t_stop; a.status = st->status; a.sum_g = st->sum_g; a.sum_g2 = st->sum_g2; a.entropy = st->entropy; a.sum_h = st->sum_h;
-  a.records = st->records; a.ticket = st->ticket; a.dev_status = st->dev_status;
-
-  a.greedy = (p->temperature == 0.f);
-  const double inv_t = a.greedy ? 1.0 : 1.0 / (double)p->temperature;
-  a.inv_temp = (float)inv_t;
-  a.k2 = (float)(inv_t * 1.4426950408889634074);
-  a.mu_g = p->mu_g;
-  a.inv_sigma = (float)(1.0 / sqrt((double)p->sigma2_g + (double)p->delta));
-  a.clip_c = p->clip_c;
-  a.alpha_s = p->alpha_s;
-  a.one_minus_alpha = 1.0f - p->alpha_s;
-  a.beta = p->beta; a.eps = p->eps;
-  a.warmup_complete = p->warmup_complete; a.t_max = p->t_max; a.eos_token = p->eos_token;
-  a.want_entropy = p->want_entropy != 0;
-  a.stop_mode = p->stop_mode; a.shadow = p->shadow != 0; a.tau = p->tau; a.p_random = p->p_random;
-  a.key0 = (uint32_t)(st->seed & 0xffffffffull);
-  a.key1 = (uint32_t)(st->seed >> 32);
-  a.batch_bits = (uint32_t)(st->batch_id << 2);
   a.tokens_out = tokens_out; a.stop_out = stop_out;
 
-  const bool bulk = ((uintptr_t)logits % 16 == 0) && (a.row_stride_bytes % 16 == 0) && (((size_t)st->V * es) % 16 == 0);
+  const bool bulk = ((uintptr_t)logits % 16 == 0) && (a.row_stride_bytes % 16 == 0) && (((size_t)v_eff * es) % 16 == 0);
   StepKernel k = pick_kernel(es, p->sampler, bulk);
   k<<<(unsigned)grid, (unsigned)(warps + fin) * 32u, smem, (cudaStream_t)stream>>>(a);
+  ESPO_CUDA_TRY(cudaGetLastError());
+  return ESPO_OK;
+}
+
+int espo_step(const void* logits, int32_t logits_dtype, int64_t row_stride, const void* values, int32_t values_dtype,
+              const int32_t* row_ids, int32_t n_rows, espo_state* st, const espo_params* p, int32_t* tokens_out,
+              uint8_t* stop_out, void* stream) {
+  if (!st) return ESPO_ERR_NULL;
+  return step_launch(logits, logits_dtype, row_stride, values, values_dtype, row_ids, n_rows, st, p, tokens_out, stop_out,
+                     st->V, 0, nullptr, stream);
+}
+
+int espo_step_partial(const void* logits_shard, int32_t logits_dtype, int64_t row_stride, int32_t v_shard,
+                      int32_t vocab_offset, const int32_t* row_ids, int32_t n_rows, espo_state* st, const espo_params* p,
+                      espo_partial* partial_out, void* stream) {
+  if (!st || !p) return ESPO_ERR_NULL;
+  if (v_shard < 1 || vocab_offset < 0 || (vocab_offset & 3) || (long long)vocab_offset + v_shard > st->V) return ESPO_ERR_BAD_SHAPE;
+  if (p->sampler != ESPO_SAMPLER_FLAT) return ESPO_ERR_BAD_PARAM;   // the flat sampler's draws belong to ids, not to blocks of a row
+  if (n_rows > 0 && !partial_out) return ESPO_ERR_NULL;
+  return step_launch(logits_shard, logits_dtype, row_stride, nullptr, ESPO_F32, row_ids, n_rows, st, p, nullptr, nullptr,
+                     v_shard, vocab_offset, partial_out, stream);
+}
+
+int espo_step_merge(const espo_partial* partials, int32_t n_shards, int64_t shard_stride, const void* values,
+                    int32_t values_dtype, const int32_t* row_ids, int32_t n_rows, espo_state* st, const espo_params* p,
+                    int32_t* tokens_out, uint8_t* stop_out, void* stream) {
+  using namespace espo;
+  if (!st || !p) return ESPO_ERR_NULL;
+  if (n_rows < 0 || n_shards < 1 || shard_stride < n_rows) return ESPO_ERR_BAD_SHAPE;
+  if (n_rows > st->capacity) return ESPO_ERR_CAPACITY;
+  if (values_dtype != ESPO_F32 && values_dtype != ESPO_BF16) return ESPO_ERR_BAD_DTYPE;
+  StepArgs a;
+  memset(&a, 0, sizeof(a));
+  {
+    const int rc = fill_params(a, st, p);
+    if (rc != ESPO_OK) return rc;
+  }
+  if (p->sampler != ESPO_SAMPLER_FLAT) return ESPO_ERR_BAD_PARAM;
+  if (n_rows == 0) return ESPO_OK;
+  if (!partials || !values || !tokens_out || !stop_out) return ESPO_ERR_NULL;
+  const int ves = (values_dtype == ESPO_BF16) ? 2 : 4;
+  if (((uintptr_t)partials % 16) || ((uintptr_t)values % ves) || ((uintptr_t)tokens_out % 4) || (row_ids && ((uintptr_t)row_ids % 4)))
+    return ESPO_ERR_ALIGN;
+  a.values = values;
+  a.values_bf16 = (values_dtype == ESPO_BF16);
+  a.row_ids = row_ids;
+  a.n_rows = n_rows; a.V = st->V;
+  a.partials = partials; a.n_shards = n_shards; a.shard_stride = shard_stride;
+  a.tokens_out = tokens_out; a.stop_out = stop_out;
+  espo_merge_kernel<<<(unsigned)((n_rows + 63) / 64), 64, 0, (cudaStream_t)stream>>>(a);
   ESPO_CUDA_TRY(cudaGetLastError());
   return ESPO_OK;
 }

@@ -46,3 +46,34 @@ def sum_over_ranks(values, dist=None, device="cpu") -> list:
     if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return t.tolist()
+
+
+# ---- vocabulary shards (tensor-parallel LM head): espo_step_partial on every rank, one all-gather, espo_step_merge ----
+
+def vocab_shards(V: int, world: int, multiple: int = 128) -> List[Tuple[int, int]]:
+    """Contiguous (offset, size) shards of the vocabulary, one per rank; every offset is a multiple of ``multiple``
+    (espo_step_partial wants a multiple of 4; 128 keeps rows of bf16 shards 256-byte aligned).  Trailing ranks may get
+    an empty shard when V is small."""
+    if world < 1 or V < 1 or multiple < 4 or multiple % 4:
+        raise ValueError("need world >= 1, V >= 1 and a shard granularity that is a multiple of 4")
+    units = (V + multiple - 1) // multiple
+    out = []
+    for r in range(world):
+        lo = min((r * units // world) * multiple, V)
+        hi = min(((r + 1) * units // world) * multiple, V)
+        out.append((lo, hi - lo))
+    return out
+
+
+def all_gather_partials(local: torch.Tensor, dist=None) -> torch.Tensor:
+    """Brings every rank's partials (float32 [rows, 8], one espo_partial per row) together as [world, rows, 8], in rank
+    order, which is the layout espo_step_merge reads.  The only data-path collective of the vocabulary-sharded step:
+    32 bytes per row and rank."""
+    if local.dim() != 2 or local.shape[1] != 8 or local.dtype != torch.float32:
+        raise ValueError("partials must be float32 [rows, 8]")
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return local.contiguous().unsqueeze(0)
+    world = dist.get_world_size()
+    out = torch.empty((world,) + tuple(local.shape), dtype=local.dtype, device=local.device)
+    dist.all_gather(list(out.unbind(0)), local.contiguous())
+    return out

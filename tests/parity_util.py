@@ -65,10 +65,14 @@ class ParityRun:
         self.check = set(range(capacity)) if check_slots is None else set(int(s) for s in check_slots)
         self.dropped = set()
         self.entropy_log = {}      # slot -> oracle entropies of its steps (when params.want_entropy)
+        self.launch = None         # callable(run, logits, values, row_ids, n) replacing espo_step
 
     def step(self, logits: torch.Tensor, values: torch.Tensor, row_ids: torch.Tensor | None = None):
         n = logits.shape[0]
-        espo.espo_step(logits, values, self.state, self.params, self.tokens, self.stop, row_ids=row_ids, n_rows=n)
+        if self.launch is None:
+            espo.espo_step(logits, values, self.state, self.params, self.tokens, self.stop, row_ids=row_ids, n_rows=n)
+        else:      # another route to the same step (the vocabulary-sharded pair of calls)
+            self.launch(self, logits, values, row_ids, n)
         torch.cuda.synchronize()
         slots = np.arange(n) if row_ids is None else row_ids[:n].cpu().numpy()
         tok = self.tokens[:n].cpu().numpy()

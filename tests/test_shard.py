@@ -35,7 +35,10 @@ def _worker(rank, world, port, out_dir):
     tot = shard.sum_over_ranks([512.0, float(rank)], dist)
     seeds = [None] * world
     dist.all_gather_object(seeds, (plan["state_seed"], plan["data_seed_offset"], plan["rows"]))
-    torch.save({"ms": ms, "tot": tot, "seeds": seeds, "plan": plan}, os.path.join(out_dir, f"r{rank}.pt"))
+    # vocabulary shards: each rank contributes its partials, everyone ends with [world, rows, 8] in rank order
+    mine = torch.full((5, 8), float(rank + 1)) + torch.arange(5, dtype=torch.float32)[:, None]
+    gathered = shard.all_gather_partials(mine, dist)
+    torch.save({"ms": ms, "tot": tot, "seeds": seeds, "plan": plan, "gathered": gathered}, os.path.join(out_dir, f"r{rank}.pt"))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -48,6 +51,21 @@ def test_two_ranks_shard_rows_and_reduce_timings(tmp_path):
         assert r["ms"] == [11.0, 5.0]                    # max over ranks, element-wise, same on every rank
         assert r["tot"] == [1024.0, 1.0]
         assert r["plan"]["global_rows"] == 1024
+        g = r["gathered"]
+        assert tuple(g.shape) == (world, 5, 8) and g.is_contiguous()
+        for k in range(world):
+            assert torch.equal(g[k], torch.full((5, 8), float(k + 1)) + torch.arange(5, dtype=torch.float32)[:, None])
     seeds = res[0]["seeds"]
     assert len({s[0] for s in seeds}) == world and len({s[1] for s in seeds}) == world   # no shared noise or data
     assert [s[2] for s in seeds] == [(0, 512), (512, 1024)]                               # disjoint, contiguous rows
+
+
+def test_vocab_shards_cover_the_vocabulary():
+    for V, w in ((152064, 8), (152064, 1), (128256, 4), (32000, 3), (1000, 8), (5, 2)):
+        parts = shard.vocab_shards(V, w)
+        assert len(parts) == w and parts[0][0] == 0 and sum(n for _, n in parts) == V
+        assert all(lo % 128 == 0 or n == 0 for lo, n in parts)
+        assert all(a[0] + a[1] == b[0] for a, b in zip(parts, parts[1:]))
+    assert shard.all_gather_partials(torch.zeros(3, 8)).shape == (1, 3, 8)      # no process group: one shard
+    with pytest.raises(ValueError):
+        shard.vocab_shards(100, 2, multiple=6)
