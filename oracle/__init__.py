@@ -47,7 +47,8 @@ class Params(C.Structure):
                 ("delta", C.c_double), ("clip_c", C.c_double), ("alpha_s", C.c_double),
                 ("beta", C.c_double), ("eps", C.c_double), ("warmup_complete", C.c_int32),
                 ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32),
-                ("stop_mode", C.c_int32), ("shadow", C.c_int32), ("tau", C.c_double), ("p_random", C.c_double)]
+                ("stop_mode", C.c_int32), ("shadow", C.c_int32), ("tau", C.c_double), ("p_random", C.c_double),
+                ("top_p", C.c_double), ("top_k", C.c_int32), ("pad_", C.c_int32)]
 
 
 class RowState(C.Structure):
@@ -60,15 +61,16 @@ class StepOut(C.Structure):
     _fields_ = [("g", C.c_double), ("g_tilde", C.c_double), ("z", C.c_double), ("logp", C.c_double),
                 ("max_x", C.c_double), ("log_s", C.c_double), ("min_rel_gap", C.c_double),
                 ("threshold", C.c_double), ("entropy", C.c_double), ("token", C.c_int32), ("stop", C.c_int32),
-                ("runner_up", C.c_int32), ("bad", C.c_int32)]
+                ("runner_up", C.c_int32), ("bad", C.c_int32), ("filter_margin", C.c_double), ("kept", C.c_int64)]
 
 
 def make_params(temperature=1.0, mu_g=0.0, sigma2_g=1.0, delta=1e-8, clip_c=10.0, alpha_s=0.9,
                 beta=7.0, eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=SAMPLER_FLAT,
-                stop_mode=0, shadow=0, tau=0.0, p_random=0.0) -> Params:
+                stop_mode=0, shadow=0, tau=0.0, p_random=0.0, top_p=1.0, top_k=0) -> Params:
     return Params(float(temperature), float(mu_g), float(sigma2_g), float(delta), float(clip_c),
                   float(alpha_s), float(beta), float(eps), int(warmup_complete), int(t_max),
-                  int(eos_token), int(sampler), int(stop_mode), int(shadow), float(tau), float(p_random))
+                  int(eos_token), int(sampler), int(stop_mode), int(shadow), float(tau), float(p_random),
+                  float(top_p), int(top_k), 0)
 
 
 def lib():

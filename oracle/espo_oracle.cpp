@@ -38,19 +38,26 @@
 //     actually sampled from.  temperature == 0 means greedy: a_t = first argmax,
 //     g_t = 0, log pi(a_t) = 0.
 //   * a sampled EOS ends the trajectory naturally even if the test would also fire.
+//   * filtered sampling (flat sampler; the paper's evaluation decodes with top-p 0.7 and says no more): a token
+//     stays in the support iff the tokens strictly more probable than it weigh less than top_p and number fewer
+//     than top_k, so tokens of equal probability stay or go together; the token is the Gumbel-max over the
+//     support with the flat sampler's draws; log pi(a_t) is taken under the renormalised support, the regret
+//     of Eq. 6 is unchanged (the normaliser cancels and the most probable token is always in the support).
 //
 //   * r_fail REPLACES the stored last reward of a stopped trajectory (Eq. 13 sets it).
 //
-// Four of these readings are fixed by nothing the paper prints, and no test can hold them to
+// Five of these readings are fixed by nothing the paper prints, and no test can hold them to
 // anything but this file's own statement -- for them parity is "parity unpinned" by the paper:
 // which distribution pi is in Eq. 6 (temperature-scaled here), the values of delta and c in
-// Eq. 9 (run-time parameters), EOS taking precedence over a stop on the same step, and
-// r_fail replacing (not adding to) the stored reward.  Everything else is pinned by the tests
+// Eq. 9 (run-time parameters), EOS taking precedence over a stop on the same step,
+// r_fail replacing (not adding to) the stored reward, and how ties at the edge of a top-p / top-k support are cut
+// (kept together here).  Everything else is pinned by the tests
 // (known-answer vectors, library routines, closed forms, invariants, brute force).
 //
 // Everything is brute force over the vocabulary, one row at a time, no blocking or
 // reordering beyond what the definitions above state.
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -169,6 +176,13 @@ struct espo_oracle_params {
   int32_t shadow;
   double tau;
   double p_random;
+  // Filtered sampling (flat sampler only; the paper's evaluation samples with top-p 0.7).  With pi the temperature-
+  // scaled softmax, token a stays in the support iff the mass of the tokens strictly more probable than a is below
+  // top_p (top_p >= 1: no filter) and fewer than top_k tokens are strictly more probable than a (top_k <= 0: no
+  // filter).  Tokens of equal probability are therefore kept or dropped together, whatever their ids.
+  double top_p;
+  int32_t top_k;
+  int32_t pad_;
 };
 
 enum { ORACLE_ACTIVE = 0, ORACLE_STOPPED = 1, ORACLE_EOS = 2, ORACLE_TMAX = 3, ORACLE_BAD = 4 };
@@ -194,6 +208,10 @@ struct espo_oracle_step_out {
   int32_t stop;
   int32_t runner_up;             // token that the closest argmax would have produced instead (-1 unknown)
   int32_t bad;                   // 1: row had NaN / +inf / no finite logit
+  // filtered sampling only: size of the support, and how far the nearest keep/drop decision was from flipping
+  // (distance of the mass above the last kept and above the first dropped value from top_p; inf without top-p)
+  double filter_margin;
+  int64_t kept;
 };
 
 void espo_oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
@@ -273,10 +291,46 @@ void espo_oracle_step_row(const double* logits, int64_t V, double value,
 
   const DrawKey dk{seed, batch_id, slot, (uint32_t)st->t};
   int64_t token = -1;
+  double filtered_log_s = out->log_s;   // log of the support's mass relative to exp(m); the whole row without a filter
+  out->filter_margin = std::numeric_limits<double>::infinity();
+  out->kept = V;
   if (forced_token >= 0) {
     token = forced_token;
   } else if (greedy) {
     token = first_argmax;
+  } else if (p->sampler == 0 && (p->top_k > 0 || p->top_p < 1.0)) {
+    // ---- support of the filtered distribution, from its definition: ids ordered by decreasing probability,
+    //      groups of equal probability taken as a whole ----
+    std::vector<int64_t> order(V);
+    for (int64_t a = 0; a < V; ++a) order[a] = a;
+    std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return x[a] > x[b] || (x[a] == x[b] && a < b); });
+    std::vector<char> keep(V, 0);
+    double mass_above = 0.0;        // probability of everything strictly more probable than the current group
+    int64_t count_above = 0;
+    double margin = std::numeric_limits<double>::infinity();
+    int64_t kept = 0;
+    for (int64_t i = 0; i < V;) {
+      int64_t j = i;
+      double group = 0.0;
+      while (j < V && x[order[j]] == x[order[i]]) { group += std::exp(x[order[j]] - m) / s; ++j; }
+      const bool in_p = (p->top_p >= 1.0) || (mass_above < p->top_p);
+      const bool in_k = (p->top_k <= 0) || (count_above < p->top_k);
+      if (p->top_p < 1.0 && x[order[i]] > NEG_INF) margin = std::fmin(margin, std::fabs(mass_above - p->top_p));
+      if (!(in_p && in_k)) break;   // every later group has at least this much above it
+      for (int64_t q = i; q < j; ++q) if (x[order[q]] > NEG_INF) { keep[order[q]] = 1; ++kept; }
+      mass_above += group;
+      count_above += j - i;
+      i = j;
+    }
+    out->filter_margin = margin;
+    out->kept = kept;
+    double s_kept = 0.0;
+    for (int64_t a = 0; a < V; ++a) if (keep[a]) s_kept += std::exp(x[a] - m);
+    filtered_log_s = std::log(s_kept);
+    ArgmaxResult r = perturbed_argmax(0, V, [&](int64_t a) { return keep[a] ? x[a] + gumbel_for(dk, 0, (uint64_t)a) : NEG_INF; });
+    token = r.index;
+    out->min_rel_gap = relative_gap(r.best, r.second);
+    out->runner_up = (int32_t)r.runner;
   } else if (p->sampler == 0) {
     ArgmaxResult r = perturbed_argmax(0, V, [&](int64_t a) { return x[a] + gumbel_for(dk, 0, (uint64_t)a); });
     token = r.index;
@@ -308,7 +362,7 @@ void espo_oracle_step_row(const double* logits, int64_t V, double value,
   // Eq. 6: the normaliser cancels in the difference of the two log-probabilities.
   const double x_tok = x[token];
   const double g = greedy ? 0.0 : (m - x_tok);
-  const double logp = greedy ? 0.0 : (x_tok - m - out->log_s);
+  const double logp = greedy ? 0.0 : (x_tok - m - filtered_log_s);   // under the distribution the token was drawn from
 
   // Eq. 9 with the frozen batch statistics.
   double gt = (g - p->mu_g) / std::sqrt(p->sigma2_g + p->delta);

@@ -463,3 +463,68 @@ def test_entropy_matches_library_and_closed_forms():
         assert abs(outs[0].entropy - stats.entropy(special.softmax(x[0] / T))) < 1e-10
         assert abs(outs[1].entropy - math.log(V)) < 1e-10
         assert outs[2].entropy == 0.0 and outs[2].token == 5
+
+
+# --------------------------------------------------------------------------- filtered sampling (top-p / top-k)
+
+
+def _support_by_brute_force(x, temperature, top_p, top_k):
+    """Token a stays iff the tokens strictly more probable than a weigh less than top_p and number fewer than top_k."""
+    q = special.softmax(np.asarray(x, dtype=np.float64) / temperature)
+    keep = np.zeros(q.size, dtype=bool)
+    for a in range(q.size):
+        above = x > x[a]
+        keep[a] = (top_p >= 1.0 or q[above].sum() < top_p) and (top_k <= 0 or int(above.sum()) < top_k) and np.isfinite(x[a])
+    return q, keep
+
+
+@pytest.mark.parametrize("top_p,top_k", [(0.7, 0), (1.0, 3), (0.9, 4), (0.35, 0), (0.999, 0)])
+def test_filtered_sampler_draws_from_the_renormalised_support(top_p, top_k):
+    # ties on purpose: ids 1 and 6 share a logit, so do 2 and 7 -- equal tokens stay or go together
+    x = np.array([1.2, 0.4, 0.0, 2.0, -1.5, 0.7, 0.4, 0.0, -np.inf, 1.9])
+    temperature = 0.8
+    q, keep = _support_by_brute_force(x, temperature, top_p, top_k)
+    slots, steps = 64, 1500
+    ro = oracle.Rollout(slots, seed=21)
+    p = oracle.make_params(temperature=temperature, sampler=oracle.SAMPLER_FLAT, warmup_complete=0, t_max=10**9,
+                           top_p=top_p, top_k=top_k)
+    rows = np.tile(x, (slots, 1))
+    counts = np.zeros(x.size, dtype=np.int64)
+    for _ in range(steps):
+        for o in ro.step(rows, np.zeros(slots), p, n_threads=8):
+            counts[o.token] += 1
+            assert o.kept == int(keep.sum())
+            want_logp = np.log(q[o.token] / q[keep].sum())
+            assert abs(o.logp - want_logp) < 1e-12 and abs(o.g - (x.max() - x[o.token]) / temperature) < 1e-12
+    assert counts[~keep].sum() == 0                                   # nothing outside the support is ever drawn
+    if keep.sum() > 1:
+        chi2, pval = stats.chisquare(counts[keep], q[keep] / q[keep].sum() * counts.sum())
+        assert pval > 1e-3, (chi2, pval)
+    if (top_p, top_k) == (0.7, 0):
+        assert list(np.nonzero(keep)[0]) == [0, 3, 9]                 # 0.37 + 0.33 < 0.7 <= 0.37 + 0.33 + 0.14
+    if (top_p, top_k) == (1.0, 3):
+        assert list(np.nonzero(keep)[0]) == [0, 3, 9]
+    if (top_p, top_k) == (0.9, 4):
+        assert list(np.nonzero(keep)[0]) == [0, 3, 5, 9]
+
+
+def test_filters_that_keep_everything_change_nothing_and_top_k_one_is_the_argmax():
+    rng = np.random.default_rng(3)
+    x = rng.normal(0, 2, size=(6, 300))
+    base = oracle.Rollout(6, seed=9).step(x, np.zeros(6), oracle.make_params(sampler=oracle.SAMPLER_FLAT))
+    same = oracle.Rollout(6, seed=9).step(x, np.zeros(6), oracle.make_params(sampler=oracle.SAMPLER_FLAT, top_p=1.0, top_k=0))
+    wide = oracle.Rollout(6, seed=9).step(x, np.zeros(6), oracle.make_params(sampler=oracle.SAMPLER_FLAT, top_p=1.0, top_k=300))
+    one = oracle.Rollout(6, seed=9).step(x, np.zeros(6), oracle.make_params(sampler=oracle.SAMPLER_FLAT, top_k=1))
+    tiny = oracle.Rollout(6, seed=9).step(x, np.zeros(6), oracle.make_params(sampler=oracle.SAMPLER_FLAT, top_p=1e-9))
+    for r in range(6):
+        assert base[r].token == same[r].token == wide[r].token and abs(base[r].logp - wide[r].logp) < 1e-12
+        assert one[r].token == tiny[r].token == int(np.argmax(x[r])) and one[r].kept == 1
+        assert abs(one[r].logp) < 1e-12 and one[r].g == 0.0           # the support is one token: probability 1, no regret
+        assert np.isinf(one[r].filter_margin) and tiny[r].filter_margin < 1.0
+
+
+def test_filter_margin_is_the_distance_of_the_nearest_decision_from_flipping():
+    x = np.log(np.array([0.5, 0.3, 0.15, 0.05]))
+    o = oracle.Rollout(1, seed=1).step(x[None, :], np.zeros(1), oracle.make_params(sampler=oracle.SAMPLER_FLAT, top_p=0.82))[0]
+    # masses above the four tokens: 0, 0.5, 0.8, 0.95 -> kept 0, 1, 2; nearest decision: |0.8 - 0.82|
+    assert o.kept == 3 and abs(o.filter_margin - 0.02) < 1e-12
