@@ -103,6 +103,14 @@ typedef struct espo_params {
   int32_t want_entropy;     /* != 0: also compute the policy entropy H(pi(.|s_t)) in the same */
                             /* pass (the quantity tracked in the analysis section); needs    */
                             /* ESPO_SAMPLER_HIER                                              */
+  /* Filtered sampling (the paper's evaluation decodes with top-p 0.7, Sec. 5; it gives no rule for ties): a token
+   * stays in the support iff the tokens strictly more probable than it weigh less than top_p and number fewer than
+   * top_k, so equally probable tokens stay or go together; the token is drawn from the renormalised support and
+   * log pi(a_t) refers to it, the regret of Eq. 6 is unchanged.  Needs ESPO_SAMPLER_FLAT; ignored when greedy.
+   * A filtered step runs its own kernel (one CTA per row, the row re-read from L2 once per 8 bits of the logit
+   * type), not the single-sweep one. */
+  float   top_p;            /* in (0, 1): nucleus mass; <= 0 or >= 1: no filter                */
+  int32_t top_k;            /* > 0: at most the k most probable (more if tied); 0: no filter  */
 } espo_params;
 
 /* Opaque per-rollout-batch state: for each of `capacity` trajectory slots the smoothed

@@ -40,15 +40,17 @@ class espo_params(C.Structure):
                 ("beta", C.c_float), ("eps", C.c_float), ("warmup_complete", C.c_int32),
                 ("t_max", C.c_int32), ("eos_token", C.c_int32), ("sampler", C.c_int32),
                 ("stop_mode", C.c_int32), ("shadow", C.c_int32), ("tau", C.c_float), ("p_random", C.c_float),
-                ("want_entropy", C.c_int32)]
+                ("want_entropy", C.c_int32), ("top_p", C.c_float), ("top_k", C.c_int32)]
 
 
 def make_params(temperature=1.0, mu_g=0.0, sigma2_g=1.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0,
                 eps=0.2, warmup_complete=1, t_max=8192, eos_token=-1, sampler=ESPO_SAMPLER_HIER,
-                stop_mode=ESPO_STOP_ESPO, shadow=0, tau=0.0, p_random=0.0, want_entropy=0) -> espo_params:
+                stop_mode=ESPO_STOP_ESPO, shadow=0, tau=0.0, p_random=0.0, want_entropy=0, top_p=1.0,
+                top_k=0) -> espo_params:
     """Defaults follow the paper's hyper-parameter table (alpha_s 0.9, beta 7.0, eps 0.2, T_max 8192)."""
     return espo_params(temperature, mu_g, sigma2_g, delta, clip_c, alpha_s, beta, eps, warmup_complete, t_max,
-                       eos_token, sampler, stop_mode, int(bool(shadow)), tau, p_random, int(bool(want_entropy)))
+                       eos_token, sampler, stop_mode, int(bool(shadow)), tau, p_random, int(bool(want_entropy)), top_p,
+                       int(top_k))
 
 
 _lib = None

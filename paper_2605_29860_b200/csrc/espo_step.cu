@@ -77,6 +77,8 @@ struct StepArgs {
   int warmup_complete, t_max, eos_token;
   int stop_mode, shadow, want_entropy;
   float tau, p_random;
+  float top_p;          // filtered sampling: < 1 keeps a nucleus (>= 1: off)
+  int top_k;            // filtered sampling: > 0 keeps the k most probable (0: off)
   uint32_t key0, key1, batch_bits;
   // outputs
   int32_t* tokens_out;
@@ -955,6 +957,394 @@ __global__ void __launch_bounds__(64) espo_merge_kernel(const __grid_constant__ 
   commit_row(a, row, pre, ds, M, S, logf(S), 0.f, x_best, best_id, true);
 }
 
+// -------------------------------------------------------------------------------------------
+// Filtered sampling (top-p / top-k, flat sampler).  A token stays in the support iff the tokens strictly more
+// probable than it weigh less than top_p and number fewer than top_k, so the support is "every logit >= tau" for
+// one threshold tau, which a radix search over the logits' bit patterns finds exactly: one pass per 8-bit digit (two
+// for bfloat16, four for float32), each a histogram of (count, probability mass) over the 256 values of the digit
+// among the logits that share the digits found so far.  Masses are summed as 2^-40 fixed point, so the sums do
+// not depend on the order of the additions and a repeated call takes the same decisions.  One CTA per row; the row
+// is read once from HBM (maximum) and then from L2 (digit passes, sampling pass).
+// -------------------------------------------------------------------------------------------
+constexpr int kFiltThreads = 1024;
+constexpr int kFiltWarps = kFiltThreads / 32;
+constexpr int kFiltSeg = 320;                      // candidate-list entries per warp
+constexpr int kFiltCopies = 16;                    // private copies of the digit histogram (two warps share one)
+constexpr size_t kFiltSmemBytes = (size_t)kFiltCopies * 256 * sizeof(uint4) +
+                                  256 * (sizeof(unsigned long long) + sizeof(unsigned)) + 192 * sizeof(float) +
+                                  (size_t)kFiltWarps * kFiltSeg * sizeof(uint2) + 128;
+
+// A probability mass e in [0, 1] as an integer count of 2^-40 (exact for a float; two 32-bit conversions).
+__device__ __forceinline__ unsigned long long filt_fixed(float e) {
+  const unsigned hi = __float2uint_rz(e * 65536.f);                       // e's first 16 binary places
+  const float rest = fmaf(-(float)hi, 1.52587890625e-05f, e);             // exact: the places that follow
+  return ((unsigned long long)hi << 24) + __float2uint_rz(rest * 1099511627776.f);
+}
+
+// Monotone key of a logit's bit pattern (larger logit, larger key); -0 and +0 share a key.
+template <int ES>
+__device__ __forceinline__ uint32_t filt_key(uint32_t bits) {
+  if (ES == 2) {
+    if (bits == 0x8000u) bits = 0u;
+    return (bits & 0x8000u) ? (~bits & 0xffffu) : (bits | 0x8000u);
+  }
+  if (bits == 0x80000000u) bits = 0u;
+  return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+
+struct FiltCross {
+  int bin;                       // first bin, from 255 down, after which a limit is reached; -1: none
+  int last;                      // lowest non-empty bin, -1: all empty
+  unsigned long long m, last_m;  // mass above `bin` / above `last`
+  unsigned c, last_c;            // count above `bin` / above `last`
+};
+
+// Walks 256 bins of (mass, count) from the top, starting from (acc_m, acc_c) above them, and finds the first bin
+// after which the mass reaches pf or the count reaches kf.  Called by one whole warp: lane l owns bins 255-8l .. 248-8l.
+__device__ __forceinline__ FiltCross filt_cross(const unsigned long long* mass, const unsigned* cnt, unsigned long long acc_m,
+                                                unsigned acc_c, unsigned long long pf, unsigned long long kf, int lane) {
+  unsigned long long lm = 0ull;
+  unsigned lc = 0u;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { lm += mass ? mass[255 - 8 * lane - i] : 0ull; lc += cnt[255 - 8 * lane - i]; }
+  unsigned long long pm = lm;
+  unsigned pc = lc;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long um = __shfl_up_sync(kFullMask, pm, o);
+    const unsigned uc = __shfl_up_sync(kFullMask, pc, o);
+    if (lane >= o) { pm += um; pc += uc; }
+  }
+  unsigned long long cm = acc_m + pm - lm;     // above this lane's bins
+  unsigned cc = acc_c + pc - lc;
+  FiltCross r{-1, -1, 0ull, 0ull, 0u, 0u};
+  for (int i = 0; i < 8; ++i) {
+    const int b = 255 - 8 * lane - i;
+    const unsigned n = cnt[b];
+    if (n == 0u) continue;
+    const unsigned long long mb = mass ? mass[b] : 0ull;
+    r.last = b; r.last_m = cm; r.last_c = cc;
+    if (r.bin < 0 && (cm + mb >= pf || (unsigned long long)cc + n >= kf)) { r.bin = b; r.m = cm; r.c = cc; }
+    cm += mb; cc += n;
+  }
+  const unsigned hit = __ballot_sync(kFullMask, r.bin >= 0), any = __ballot_sync(kFullMask, r.last >= 0);
+  const int fl = hit ? __ffs(hit) - 1 : 0, ll = any ? 31 - __clz(any) : 0;
+  FiltCross out;
+  out.bin = hit ? __shfl_sync(kFullMask, r.bin, fl) : -1;
+  out.m = __shfl_sync(kFullMask, r.m, fl);
+  out.c = __shfl_sync(kFullMask, r.c, fl);
+  out.last = any ? __shfl_sync(kFullMask, r.last, ll) : -1;
+  out.last_m = __shfl_sync(kFullMask, r.last_m, ll);
+  out.last_c = __shfl_sync(kFullMask, r.last_c, ll);
+  return out;
+}
+
+template <int ES>
+__global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __grid_constant__ StepArgs a) {
+  extern __shared__ __align__(16) unsigned char fsm[];
+  // digit histograms: per bin the mass as three limbs of 14 + 13 + 13 bits (32-bit shared-memory atomics are native,
+  // 64-bit ones are not; a copy sees fewer than 2^18 logits per pass, so no limb overflows) and the count
+  uint4* whist = reinterpret_cast<uint4*>(fsm);                                          // [copies][256]
+  unsigned long long* bmass = reinterpret_cast<unsigned long long*>(whist + kFiltCopies * 256);   // [256] all copies together
+  unsigned* bcnt = reinterpret_cast<unsigned*>(bmass + 256);                             // [256]
+  float* red_f = reinterpret_cast<float*>(bcnt + 256);                                   // [32] scores / sums
+  int* red_i = reinterpret_cast<int*>(red_f + 32);                                       // [32] ids, flags
+  unsigned long long* red_u = reinterpret_cast<unsigned long long*>(red_i + 32);         // [2][32] integer sums
+  uint2* cand = reinterpret_cast<uint2*>(red_u + 64);                                    // [warps][kFiltSeg] (id, bits)
+  unsigned* sbin = reinterpret_cast<unsigned*>(whist);                                   // 4096 sample bins (before the digit passes)
+  __shared__ RowPre pre_s;
+  __shared__ unsigned long long sh_acc_mass, sh_kept_mass;
+  __shared__ unsigned sh_acc_cnt, sh_prefix, sh_cut_a;
+  __shared__ int sh_found, sh_overflow;
+  __shared__ unsigned seg_n[kFiltWarps];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float NINF = __int_as_float(0xff800000);
+  constexpr int VEC = 16 / ES;
+
+  for (int row = blockIdx.x; row < a.n_rows; row += gridDim.x) {
+    __syncthreads();                                         // the previous row's shared values are no longer read
+    if (tid == 0) { pre_s = prefetch_row(a, row); sh_overflow = 0; sh_cut_a = 0u; }
+    if (tid < kFiltWarps) seg_n[tid] = 0u;
+    for (int i = tid; i < 4096; i += kFiltThreads) sbin[i] = 0u;
+    __syncthreads();
+    const RowPre pre = pre_s;
+    if (pre.slot < 0) { mark_row(a, row, 0, tid, -1, ESPO_DEV_BAD_SLOT, -1, true); continue; }
+    if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, pre.slot, tid, -1, 0u, -1, true); continue; }   // finished: untouched
+
+    const unsigned char* row_base = a.logits + (size_t)row * a.row_stride_bytes;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(row_base) & 15u) == 0;
+    // Calls fn(id, raw bits) for every logit of the row; 16-byte loads where the row allows them.
+    auto for_each = [&](auto&& fn) {
+      const int v_main = vec_ok ? (a.V / VEC) * VEC : 0;
+      constexpr int kInFlight = 4;                           // loads a thread issues before it looks at the first
+      for (int base0 = tid * VEC; base0 < v_main; base0 += kInFlight * kFiltThreads * VEC) {
+        uint4 q[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+          const int base = base0 + u * kFiltThreads * VEC;
+          q[u] = (base < v_main) ? __ldg(reinterpret_cast<const uint4*>(row_base + (size_t)base * ES)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+          const int base = base0 + u * kFiltThreads * VEC;
+          if (base >= v_main) break;
+          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (ES == 2) { fn(base + 2 * j, w[j] & 0xffffu); fn(base + 2 * j + 1, w[j] >> 16); }
+            else fn(base + j, w[j]);
+          }
+        }
+      }
+      for (int id = v_main + tid; id < a.V; id += kFiltThreads) {
+        const uint32_t bits = (ES == 2) ? (uint32_t)__ldg(reinterpret_cast<const unsigned short*>(row_base) + id)
+                                        : __ldg(reinterpret_cast<const uint32_t*>(row_base) + id);
+        fn(id, bits);
+      }
+    };
+    auto value_of = [&](uint32_t bits) -> float { return __uint_as_float(ES == 2 ? bits << 16 : bits); };
+    // The two passes over the whole row work on groups of VEC consecutive logits, already as floats: fn(first id,
+    // values); positions past the row's end read as -inf, which no pass counts.
+    auto for_each_group = [&](auto&& fn) {
+      const int v_main = vec_ok ? (a.V / VEC) * VEC : 0;
+      constexpr int kInFlight = 4;
+      for (int base0 = tid * VEC; base0 < v_main; base0 += kInFlight * kFiltThreads * VEC) {
+        uint4 q[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+          const int base = base0 + u * kFiltThreads * VEC;
+          q[u] = (base < v_main) ? __ldg(reinterpret_cast<const uint4*>(row_base + (size_t)base * ES)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+          const int base = base0 + u * kFiltThreads * VEC;
+          if (base >= v_main) break;
+          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+          float x[VEC];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (ES == 2) { x[2 * j] = __uint_as_float(w[j] << 16); x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
+            else x[j] = __uint_as_float(w[j]);
+          }
+          fn(base, x);
+        }
+      }
+      for (int base = v_main + tid * VEC; base < a.V; base += kFiltThreads * VEC) {
+        float x[VEC];
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) x[j] = (base + j < a.V) ? load_logit<ES>(row_base, base + j) : NINF;
+        fn(base, x);
+      }
+    };
+    auto bits_of = [&](float x) -> uint32_t { return ES == 2 ? __float_as_uint(x) >> 16 : __float_as_uint(x); };
+
+    // ---- candidate cut.  A histogram of the whole row would put nearly every logit into a handful of bins, and
+    //      shared-memory atomics on one address serialise.  So 4096 logits (16 stretches of 256 spread over the row)
+    //      are sampled into a histogram over the upper 12 bits of their keys, and the cut is the key above which
+    //      64 samples lie -- about 2400 logits of the row.  The pass over the row lists the logits above the cut;
+    //      if they already reach top_p or top_k they contain the whole support and the search below runs over the
+    //      list, otherwise (or if the list overflows) it runs over the whole row again. ----
+    if (a.V >= 16384) {
+      constexpr int kStretch = 256, kStretches = 16;
+#pragma unroll
+      for (int j = 0; j < kStretch * kStretches / kFiltThreads; ++j) {
+        const int n = tid + j * kFiltThreads;                // sample number
+        const int id = (int)((long long)(n / kStretch) * a.V / kStretches) + (n % kStretch);
+        atomicAdd(sbin + (filt_key<ES>(bits_of(load_logit<ES>(row_base, id))) >> (8 * ES - 12)), 1u);
+      }
+      __syncthreads();
+      if (tid < 256) {                                       // groups of 16 bins
+        unsigned t = 0u;
+        for (int i = 0; i < 16; ++i) t += sbin[tid * 16 + i];
+        bcnt[tid] = t;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        const unsigned long long want = 64ull;
+        const FiltCross g = filt_cross(nullptr, bcnt, 0ull, 0u, ~0ull, want, lane);
+        if (lane == 0 && g.bin >= 0) {
+          unsigned cum = g.c, edge = (unsigned)(g.bin * 16);
+          for (int i = 15; i >= 0; --i) {
+            cum += sbin[g.bin * 16 + i];
+            if (cum >= want) { edge = (unsigned)(g.bin * 16 + i); break; }
+          }
+          sh_cut_a = edge << (8 * ES - 12);                  // the bin's lower edge
+        }
+      }
+    }
+    __syncthreads();
+    const uint32_t cut_a = sh_cut_a;
+    // the cut as a logit: keys are monotone in the value, so key >= cut_a is x >= cut_x
+    const uint32_t key_top = (ES == 2) ? 0x8000u : 0x80000000u;
+    const float cut_x = (cut_a == 0u) ? __int_as_float(0x7f800000)
+                                      : value_of((cut_a & key_top) ? (cut_a & ~key_top) : (~cut_a & (ES == 2 ? 0xffffu : 0xffffffffu)));
+
+    // ---- the pass over the row (from HBM): the largest logit and the row's mass sum_a exp((x_a - M)/T), kept per
+    //      thread relative to the thread's own running maximum; NaN or +inf anywhere makes the row unusable (either
+    //      turns the thread's sum into NaN or its maximum into +inf); logits at or above the cut go onto the list. ----
+    float m = NINF, s_t = 0.f;
+    uint2* my_seg = cand + warp * kFiltSeg;
+    for_each_group([&](int base, const float (&x)[VEC]) {
+      float vm = x[0];
+#pragma unroll
+      for (int j = 1; j < VEC; ++j) vm = fmaxf(vm, x[j]);
+      if (vm > m) { s_t *= ex2_approx((m - vm) * a.k2); m = vm; }   // m = -inf: s_t is 0 and stays 0
+      if (m > NINF) {
+        const float c0 = -m * a.k2;
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) s_t += ex2_approx(fmaf(x[j], a.k2, c0));   // NaN stays NaN; +inf makes m +inf, then NaN
+      } else {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) if (x[j] != x[j]) s_t = x[j];             // a NaN among logits that are all -inf so far
+      }
+      if (vm >= cut_x) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+          if (!(x[j] >= cut_x)) continue;
+          const unsigned at = atomicAdd(&seg_n[warp], 1u);
+          if (at < (unsigned)kFiltSeg) my_seg[at] = make_uint2((unsigned)(base + j), bits_of(x[j]));
+          else sh_overflow = 1;
+        }
+      }
+    });
+    bool poisoned = (s_t != s_t) || (m == __int_as_float(0x7f800000));
+    const float wm = warp_max(m);
+    poisoned = __any_sync(kFullMask, poisoned);
+    if (lane == 0) { red_f[warp] = wm; red_i[warp] = poisoned; }
+    __syncthreads();
+    float M = NINF;
+    for (int w = 0; w < kFiltWarps; ++w) { M = fmaxf(M, red_f[w]); poisoned |= red_i[w] != 0; }
+    if (poisoned || !(M > NINF)) { mark_row(a, row, pre.slot, tid, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true); continue; }
+    float tot_f = (m > NINF) ? s_t * ex2_approx((m - M) * a.k2) : 0.f;
+    tot_f = warp_sum(tot_f);                                 // fixed order: the same bits on every call
+
+    // ---- what the list holds: exact integer sums of mass and count ----
+    unsigned long long m_a = 0ull;
+    unsigned c_a = 0u;
+    if (cut_a != 0u && sh_overflow == 0) {
+      const unsigned n = seg_n[warp];
+      for (unsigned i = lane; i < n; i += 32) { m_a += filt_fixed(ex2_approx((value_of(my_seg[i].y) - M) * a.k2)); ++c_a; }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) { m_a += __shfl_xor_sync(kFullMask, m_a, o); c_a += __shfl_xor_sync(kFullMask, c_a, o); }
+    __syncthreads();
+    if (lane == 0) { red_f[warp] = tot_f; red_u[warp] = m_a; red_u[32 + warp] = c_a; }
+    __syncthreads();
+    double tot = 0.0;
+    unsigned long long ma = 0ull, ca = 0ull;                 // integer sums: the order does not matter
+    for (int w = 0; w < kFiltWarps; ++w) { tot += (double)red_f[w]; ma += red_u[w]; ca += red_u[32 + w]; }
+    const unsigned long long total = (unsigned long long)(tot * 1099511627776.0);
+    const unsigned long long pf = (a.top_p < 1.f) ? (unsigned long long)((double)total * (double)a.top_p) : ~0ull;   // top_p of the row's mass
+    const unsigned long long kf = a.top_k > 0 ? (unsigned long long)a.top_k : ~0ull;
+    const bool use_list = cut_a != 0u && (ma >= pf || ca >= kf) && sh_overflow == 0;
+    const bool cut_active = use_list;
+    // Calls fn(id, raw bits) for every logit that can belong to the support.
+    auto for_each_candidate = [&](auto&& fn) {
+      if (use_list) {
+        const unsigned n = seg_n[warp];
+        for (unsigned i = lane; i < n; i += 32) { const uint2 c = my_seg[i]; fn((int)c.x, c.y); }
+      } else {
+        for_each(fn);
+      }
+    };
+
+    // ---- digit passes: find the threshold key.  The keys that take part lie between key_lo (the cut, or 0) and
+    //      the key of the largest logit; only the bits in which that range varies are searched, 8 at a time from the
+    //      top, so the logits of a list (a narrow range of values) spread over the bins of a single pass or two. ----
+    const uint32_t key_lo = use_list ? cut_a : 0u;
+    const uint32_t span = filt_key<ES>(bits_of(M)) - key_lo;
+    const int n_digits = span == 0u ? 1 : (32 - __clz(span) + 7) / 8;
+    if (tid == 0) { sh_acc_mass = 0ull; sh_acc_cnt = 0u; sh_prefix = 0u; sh_kept_mass = total; sh_found = 0; }
+    for (int d = 0; d < n_digits; ++d) {
+      const int shift = 8 * (n_digits - 1 - d);
+      const int copies = use_list ? 4 : kFiltCopies;         // a short list needs few copies, and they cost to clear and add up
+      for (int i = tid; i < copies * 256; i += kFiltThreads) whist[i] = make_uint4(0u, 0u, 0u, 0u);
+      __syncthreads();
+      const uint32_t prefix = sh_prefix;                     // the digits above this one, as found so far
+      unsigned* my_hist = reinterpret_cast<unsigned*>(whist + (warp % copies) * 256);
+      for_each_candidate([&](int, uint32_t bits) {
+        const uint32_t key = filt_key<ES>(bits) - key_lo;    // every candidate's key is at least key_lo
+        if (d > 0 && (key >> (shift + 8)) != prefix) return;
+        const unsigned long long fx = filt_fixed(ex2_approx((value_of(bits) - M) * a.k2));
+        unsigned* h = my_hist + 4u * ((key >> shift) & 255u);
+        atomicAdd(h, (unsigned)(fx >> 26));                  // 14 bits (an e of exactly 1 gives 2^14)
+        atomicAdd(h + 1, (unsigned)(fx >> 13) & 0x1fffu);
+        atomicAdd(h + 2, (unsigned)fx & 0x1fffu);
+        atomicAdd(h + 3, 1u);
+      });
+      __syncthreads();
+      if (tid < 256) {
+        unsigned long long tm = 0ull;
+        unsigned tc = 0u;
+        for (int w = 0; w < copies; ++w) {
+          const uint4 h = whist[w * 256 + tid];
+          tm += ((unsigned long long)h.x << 26) + ((unsigned long long)h.y << 13) + h.z;
+          tc += h.w;
+        }
+        bmass[tid] = tm; bcnt[tid] = tc;
+      }
+      __syncthreads();
+      if (warp == 0 && (d == 0 || sh_found)) {
+        // Every value of a bin has at least the running mass and count above it; the first bin after which one of
+        // the two limits is reached holds the last value that stays.
+        const FiltCross x = filt_cross(bmass, bcnt, sh_acc_mass, sh_acc_cnt, pf, kf, lane);
+        int boundary = x.bin;
+        unsigned long long cum_m = x.m;
+        unsigned cum_c = x.c;
+        // a cut was enough, or an upper digit found a boundary: the boundary lies among what was histogrammed (exact
+        // sums make this branch unreachable; it keeps the search well-defined regardless)
+        if (boundary < 0 && (d > 0 || cut_active) && x.last >= 0) { boundary = x.last; cum_m = x.last_m; cum_c = x.last_c; }
+        if (lane == 0) {
+          if (boundary >= 0) {
+            sh_found = 1;
+            sh_acc_mass = cum_m; sh_acc_cnt = cum_c;
+            sh_prefix = (sh_prefix << 8) | (unsigned)boundary;
+            if (d == n_digits - 1) sh_kept_mass = cum_m + bmass[boundary];   // the boundary value itself stays
+          } else {
+            sh_found = 0;                                    // neither limit is reached: the whole row stays
+          }
+        }
+      }
+      __syncthreads();
+      if (!sh_found) break;                                  // the same for every thread: read after the barrier
+    }
+    const bool filtered = sh_found != 0;
+    const uint32_t tau_key = filtered ? key_lo + sh_prefix : 0u;   // keep everything unless a boundary was found
+    const unsigned long long kept_mass = sh_kept_mass;
+
+    // ---- sampling pass: Gumbel-max over the support with the flat sampler's draws ----
+    const DrawStream ds{a.key0, a.key1, (uint32_t)pre.t_now, (uint32_t)pre.slot, a.batch_bits};
+    float best = NINF;
+    int best_id = -1;
+    auto offer = [&](int id, uint32_t bits) {
+      if (filt_key<ES>(bits) < tau_key) return;
+      const float x = value_of(bits);
+      if (!(x > NINF)) return;
+      const float sc = fmaf(x - M, a.inv_temp, gumbel_at(ds, 0u, (uint32_t)id));
+      if (sc > best || (sc == best && id < best_id)) { best = sc; best_id = id; }
+    };
+    for_each_candidate(offer);
+    warp_argmax(best, best_id);
+    __syncthreads();                                         // red_f / red_i of the sums above are no longer read
+    if (lane == 0) { red_f[warp] = best; red_i[warp] = best_id; }
+    __syncthreads();
+    if (tid == 0) {
+      float b = NINF;
+      int tok = -1;
+      for (int w = 0; w < kFiltWarps; ++w)
+        if (red_i[w] >= 0 && (tok < 0 || red_f[w] > b || (red_f[w] == b && red_i[w] < tok))) { b = red_f[w]; tok = red_i[w]; }
+      if (tok < 0) {
+        mark_row(a, row, pre.slot, 0, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true);
+      } else {
+        const float l_tok = load_logit<ES>(row_base, tok);
+        const float S = (float)((double)kept_mass * (1.0 / 1099511627776.0));
+        commit_row(a, row, pre, ds, M, S, logf(S), 0.f, l_tok, tok, true);
+      }
+    }
+  }
+}
+
 }  // namespace espo
 
 // ===========================================================================================
@@ -1175,6 +1565,9 @@ static int fill_params(espo::StepArgs& a, const espo_state* st, const espo_param
       !(p->p_random >= 0.f && p->p_random <= 1.f))
     return ESPO_ERR_BAD_PARAM;
   if (p->want_entropy && p->sampler != ESPO_SAMPLER_HIER) return ESPO_ERR_BAD_PARAM;   // the flat sampler's records are full
+  if (isnan(p->top_p) || p->top_k < 0) return ESPO_ERR_BAD_PARAM;
+  a.top_p = (p->top_p > 0.f && p->top_p < 1.f) ? p->top_p : 1.f;
+  a.top_k = p->top_k;
   a.capacity = st->capacity;
   a.z = st->z; a.g = st->g; a.g_tilde = st->g_tilde; a.logp = st->logp;
   a.t = st->t; a.t_stop = st->t_stop; a.status = st->status; a.sum_g = st->sum_g; a.sum_g2 = st->sum_g2; a.entropy = st->entropy; a.sum_h = st->sum_h;
@@ -1282,6 +1675,21 @@ static int step_launch(const void* logits, int32_t logits_dtype, int64_t row_str
 
   a.tokens_out = tokens_out; a.stop_out = stop_out;
 
+  if (!a.greedy && (a.top_p < 1.f || a.top_k > 0)) {
+    // filtered sampling: its own kernel, one CTA per row
+    if (p->sampler != ESPO_SAMPLER_FLAT || partial_out) return ESPO_ERR_BAD_PARAM;
+    if (v_eff > (1 << 21)) return ESPO_ERR_CAPACITY;       // the histogram limbs are sized for rows up to 2^21 logits
+    static bool attr_set[2] = {false, false};
+    auto fk = (es == 2) ? espo_filtered_kernel<2> : espo_filtered_kernel<4>;
+    if (!attr_set[es == 2]) {
+      ESPO_CUDA_TRY(cudaFuncSetAttribute((const void*)fk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFiltSmemBytes));
+      attr_set[es == 2] = true;
+    }
+    const int fgrid = n_rows < st->sm_count ? n_rows : st->sm_count;
+    fk<<<(unsigned)fgrid, kFiltThreads, kFiltSmemBytes, (cudaStream_t)stream>>>(a);
+    ESPO_CUDA_TRY(cudaGetLastError());
+    return ESPO_OK;
+  }
   const bool bulk = ((uintptr_t)logits % 16 == 0) && (a.row_stride_bytes % 16 == 0) && (((size_t)v_eff * es) % 16 == 0);
   StepKernel k = pick_kernel(es, p->sampler, bulk);
   k<<<(unsigned)grid, (unsigned)(warps + fin) * 32u, smem, (cudaStream_t)stream>>>(a);

@@ -39,7 +39,8 @@ def to_oracle_params(p: espo.espo_params) -> oracle.Params:
     return oracle.make_params(temperature=p.temperature, mu_g=p.mu_g, sigma2_g=p.sigma2_g, delta=p.delta,
                               clip_c=p.clip_c, alpha_s=p.alpha_s, beta=p.beta, eps=p.eps,
                               warmup_complete=p.warmup_complete, t_max=p.t_max, eos_token=p.eos_token,
-                              sampler=p.sampler, stop_mode=p.stop_mode, shadow=p.shadow, tau=p.tau, p_random=p.p_random)
+                              sampler=p.sampler, stop_mode=p.stop_mode, shadow=p.shadow, tau=p.tau, p_random=p.p_random,
+                              top_p=(p.top_p if 0.0 < p.top_p < 1.0 else 1.0), top_k=p.top_k)
 
 
 def close(gpu: float, ref: float) -> bool:

@@ -60,4 +60,4 @@ def test_python_binding_mirrors_the_abi():
         if name == "espo_strerror" or name == "espo_last_cuda_error":
             continue
         assert hasattr(espo, name), f"binding lacks {name}"
-    assert ctypes.sizeof(espo.espo_params) == 68
+    assert ctypes.sizeof(espo.espo_params) == 76
