@@ -430,6 +430,38 @@ def main():
                                  "note": f"capacity {B} slots, bf16, V={V}; eager launches; compaction is a separate one-CTA kernel"}
             espo.espo_free_state(sst)
 
+        # ---- the other routes through the step: flat sampler, top-p filter, vocabulary shards (eager launches) ----
+        if not args.no_sweep:
+            def step_us(p, reps, fn=None):
+                sst = espo.espo_init_state(B, V, seed=5)
+                call = fn or (lambda i: espo.espo_step(bufs[i % N_BUFFERS], values, sst, p, tokens, stop))
+                for i in range(3):
+                    call(i) if fn is None else fn(i, sst)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(reps):
+                    call(i) if fn is None else fn(i, sst)
+                e1.record()
+                torch.cuda.synchronize()
+                espo.espo_free_state(sst)
+                return e0.elapsed_time(e1) * 1e3 / reps
+            flat = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, **PARAMS)
+            top_p = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, top_p=0.7, **PARAMS)
+            cuts = shard.vocab_shards(V, 8)
+            lo, n_ids = cuts[3]
+            shard_bufs = [synth.logits_batch(B, n_ids, dtype=torch.bfloat16, sd=3.0, seed=700 + i, device=dev) for i in range(16)]
+            parts = torch.zeros(8, B, 8, dtype=torch.float32, device=dev)
+            out["other_routes"] = {
+                "flat_sampler_us": step_us(flat, 20),
+                "top_p_0.7_us": step_us(top_p, 40),
+                "vocab_shard_partial_us": step_us(flat, 100, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, flat, parts[3])),
+                "vocab_shard_merge_us": step_us(flat, 100, lambda i, sst: espo.espo_step_merge(parts, values, sst, flat, tokens, stop)),
+                "note": f"same batch (B={B}, V={V}, bf16); partial: one of 8 shards ({n_ids} ids) as its own buffer; merge: 8 x {B} "
+                        f"partials (host-bound when launched eagerly from Python)",
+            }
+            del shard_bufs
+
         # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region ----
         host_logits = [torch.empty(B, V, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
         for i in range(2):
