@@ -261,6 +261,8 @@ int espo_state_status(espo_state* st, uint32_t* host_out, void* stream);
  * With r'_t the (possibly replaced) rewards and V_L := 0 for every trajectory (nothing is
  * bootstrapped past the last token): delta_t = r'_t + gamma V_{t+1} - V_t and
  * A_t = delta_t + gamma*lambda*A_{t+1}, A_L := 0.
+ * Trajectories do not interact: a NaN or infinity among one trajectory's rewards or values
+ * spoils that trajectory's advantages only.
  * Uses a per-device workspace that grows on demand: a call that needs more than any
  * earlier call (or espo_advantages_reserve) allocates device memory after synchronising
  * the device; otherwise nothing is allocated.  Calls on one device must not overlap.

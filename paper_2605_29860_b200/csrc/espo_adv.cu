@@ -167,8 +167,15 @@ static void set_discount(AdvArgs& a, float gamma, float lambda) {
 struct Map {   // X -> b + a * X
   double a, b;
 };
-// `lo` is applied after `hi` (lo belongs to the earlier tokens): lo(hi(X)).
-__device__ __forceinline__ Map compose(const Map& lo, const Map& hi) { return Map{lo.a * hi.a, fma(lo.a, hi.b, lo.b)}; }
+// `lo` is applied after `hi` (lo belongs to the earlier tokens): lo(hi(X)).  A map that contains a trajectory end
+// (a == 0) ignores its argument outright, so that a NaN or infinity in a later trajectory cannot reach an earlier one
+// through 0 * NaN.
+__device__ __forceinline__ Map compose(const Map& lo, const Map& hi) {
+  const bool cut = (lo.a == 0.0);
+  return Map{cut ? 0.0 : lo.a * hi.a, cut ? lo.b : fma(lo.a, hi.b, lo.b)};
+}
+// The value of `m` at X, with the same rule.
+__device__ __forceinline__ double apply(const Map& m, double x) { return m.a == 0.0 ? m.b : fma(m.a, x, m.b); }
 
 __device__ __forceinline__ double shfl_down_d(double v, int o) { return __shfl_down_sync(kFullMask, v, o); }
 __device__ __forceinline__ double shfl_up_d(double v, int o) { return __shfl_up_sync(kFullMask, v, o); }
@@ -530,11 +537,11 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     const double carry_in = carry_buf[par];
     if (tid == 0) {
       const Map whole = compose(m, after);
-      carry_buf[par ^ 1] = fma(whole.a, carry_in, whole.b);     // what follows the next (lower) chunk
+      carry_buf[par ^ 1] = apply(whole, carry_in);              // what follows the next (lower) chunk
     }
 
     // ---- replay the thread's tokens with the value that follows them ----
-    double x = fma(after.a, carry_in, after.b);
+    double x = apply(after, carry_in);
     float out[kAdvPerThread];
     const bool whole_thread = (q0 >= q_lo && q0 + kAdvPerThread <= q_hi);
     if (!__any_sync(kFullMask, last_mask != 0u)) {

@@ -183,3 +183,21 @@ def test_padded_layout(B, t_max, lo):
     espo.espo_advantages_padded(torch.nan_to_num(r), torch.nan_to_num(v), bad, s, 1.0, 0.95, -1.0, adv)
     torch.cuda.synchronize()
     assert espo.espo_advantages_status() & espo.ESPO_DEV_BAD_LENGTHS
+
+
+def test_a_broken_trajectory_does_not_reach_its_neighbours():
+    # NaN and infinities inside one trajectory: every other trajectory comes out as if it were not there
+    r, v, L, s = synth.ragged_trajectories(200, len_lo=1, len_hi=3000, seed=12)
+    off = torch.cumsum(L.long(), 0) - L.long()
+    for bad, val in ((17, float("nan")), (90, float("inf")), (150, float("-inf"))):
+        v[off[bad] + L[bad].long() // 2] = val
+        r[off[bad]] = val
+    adv = torch.empty_like(r)
+    espo.espo_advantages(r, v, L, s, 1.0, 0.95, -1.0, adv)
+    torch.cuda.synchronize()
+    ref = oracle.advantages(r.cpu().numpy(), v.cpu().numpy(), L.cpu().numpy(), s.cpu().numpy(), 1.0, float(np.float32(0.95)), -1.0)
+    got = adv.cpu().numpy().astype(np.float64)
+    finite = np.isfinite(ref)
+    assert finite.sum() > 0.95 * ref.size                      # the oracle keeps the damage inside the three trajectories
+    assert np.all(np.abs(got[finite] - ref[finite]) <= 1e-5 + 1e-4 * np.abs(ref[finite]))
+    assert not np.any(np.isfinite(got[~finite]))               # and what is broken stays broken
