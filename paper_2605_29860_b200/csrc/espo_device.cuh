@@ -140,18 +140,6 @@ __device__ __forceinline__ uint32_t pick_word(const uint4& w, uint32_t i) {
   return i == 0 ? w.x : (i == 1 ? w.y : (i == 2 ? w.z : w.w));
 }
 
-// 23 random bits k -> u = (2k+1)/2^24 in (0,1), exact in float32; G = -log(-log u), full-precision logs.
-__device__ __forceinline__ float gumbel_from_word(uint32_t word) {
-  const float u = __uint2float_rn(2u * (word >> 9) + 1u) * 5.9604644775390625e-08f;
-  return -logf(-logf(u));
-}
-
-// The same uniform as a standard exponential draw E = -ln u > 0 (the Gumbel is -ln E).
-__device__ __forceinline__ float expo_from_word(uint32_t word) {
-  const float u = __uint2float_rn(2u * (word >> 9) + 1u) * 5.9604644775390625e-08f;
-  return -logf(u);
-}
-
 // ln E of an exponential draw E = -ln u in [6e-8, 17]: the Gumbel is -ln E.  E itself comes from the precise
 // logf (u close to 1 makes E tiny, and its relative accuracy is what the large Gumbels rest on); its logarithm
 // may be lg2.approx: absolute error below 2^-22 for E in (0.5, 2), relative error below 2^-22 elsewhere, i.e.
@@ -160,6 +148,19 @@ __device__ __forceinline__ float ln_expo(float e) {
   float y;
   asm("lg2.approx.f32 %0, %1;" : "=f"(y) : "f"(e));
   return y * 0.6931471805599453f;
+}
+
+// 23 random bits k -> u = (2k+1)/2^24 in (0,1), exact in float32; G = -log(-log u): the inner logarithm in full
+// precision, the outer one as ln_expo.
+__device__ __forceinline__ float gumbel_from_word(uint32_t word) {
+  const float u = __uint2float_rn(2u * (word >> 9) + 1u) * 5.9604644775390625e-08f;
+  return -ln_expo(-logf(u));
+}
+
+// The same uniform as a standard exponential draw E = -ln u > 0 (the Gumbel is -ln E).
+__device__ __forceinline__ float expo_from_word(uint32_t word) {
+  const float u = __uint2float_rn(2u * (word >> 9) + 1u) * 5.9604644775390625e-08f;
+  return -logf(u);
 }
 
 // Which Philox stream a draw belongs to: (step, slot, batch|level) are counter words 1..3.
