@@ -484,6 +484,27 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
 #pragma unroll
       for (int h = 0; h < 10; ++h) w_round *= w_round;
       static_assert(4 * kAdvThreads == 1024, "w_round is the 1024th power");
+      if (a.gamma == 1.0 && a.gl == 1.0) {
+        // gamma = lambda = 1: the TD errors telescope, sum_k delta_k = sum_k r'_k - V(first token); only the rewards of
+        // the rest of the trajectory are read
+#pragma unroll 4
+        for (long long k0 = t_hi + 4 * tid; k0 < end; k0 += 4 * kAdvThreads) {
+          float r[4];
+          if (k0 + 4 <= a.total) {
+            const float4 rr = __ldg(reinterpret_cast<const float4*>(a.rewards + k0));
+            r[0] = rr.x; r[1] = rr.y; r[2] = rr.z; r[3] = rr.w;
+          } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) r[e] = (k0 + e < a.total) ? __ldg(a.rewards + k0 + e) : 0.f;
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const long long k = k0 + e;
+            if (k < end) part += (k == t_end - 1 && failed) ? r_fail_d : (double)r[e];
+          }
+        }
+        if (tid == 0) part -= (double)__ldg(a.values + t_hi);
+      } else
 #pragma unroll 4
       for (long long k0 = t_hi + 4 * tid; k0 < end; k0 += 4 * kAdvThreads, wt *= w_round) {
         float r[4], v[5];
