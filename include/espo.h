@@ -311,8 +311,8 @@ int espo_advantages_status(uint32_t* host_out, void* stream);
  *                    clamped
  *   adv_out          device float32 [B * t_max]; padding entries are written as 0
  *   returns_out      device float32 [B * t_max] or NULL; padding entries are written as 0
- * The pass reads and writes all B * t_max entries (12 bytes each, 16 with returns), padding included; a batch that is
- * mostly padding is cheaper packed.  Workspace and errors as for espo_advantages. */
+ * The pass writes all B * t_max entries and reads all but the 3072-entry chunks that lie wholly inside one row's
+ * padding; a batch that is mostly padding is cheaper packed.  Workspace and errors as for espo_advantages. */
 int espo_advantages_padded(const float* rewards, const float* values, const int32_t* lengths,
                            const uint8_t* stopped, int32_t B, int32_t t_max,
                            float gamma, float lambda, float r_fail, float* adv_out,

@@ -210,6 +210,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
   __shared__ int halo_traj;                                  // trajectory that crosses the range's upper end, or -1,
   __shared__ long long halo_end;                             // its end offset
   __shared__ int halo_failed;                                // and whether it was stopped
+  __shared__ int all_pad[kAdvStages];                        // padded layout: the stage's chunk is padding only, nothing was copied
   __shared__ int is_last_cta;                                // statistics: this CTA adds up every CTA's partial sums
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -256,6 +257,21 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
       float* vs = vbuf + stage * kAdvVStride;
       const bool tail16 = (p0 + kAdvChunk + 4 <= a.total);               // the 16 bytes after the chunk exist
       const uint32_t bytes = n4 > skip ? (uint32_t)sizeof(float) * (uint32_t)(n4 - skip) : 0u;
+      if (PADDED) {
+        // A chunk that lies wholly in one row's padding is not read at all: its padding bits make the scanning
+        // threads write zeros whatever the stage still holds.
+        const long long p_lo = max(p0, t_lo), p_end = min(p0 + kAdvChunk, a.total);
+        const long long i = p_lo / a.t_max;
+        if (p_end <= (i + 1) * a.t_max) {
+          const int len = a.lengths[i];
+          if (p_lo >= i * a.t_max + (len < 0 ? 0 : (len > a.t_max ? a.t_max : len))) {
+            all_pad[stage] = 1;                                            // published by the arrivals on full[stage]
+            mbar_arrive_expect_tx(&full[stage], 0u);
+            return;
+          }
+        }
+        all_pad[stage] = 0;
+      }
       fence_proxy_async();                                               // the scanning threads' reads of the stage come first
       mbar_arrive_expect_tx(&full[stage], 2u * bytes + (tail16 ? 16u : 0u));
       if (bytes) {
@@ -376,6 +392,20 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     const float* vs = vbuf + stage * kAdvVStride;
     const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
     if (!mbar_wait_bounded(&full[stage], (uint32_t)((k / kAdvStages) & 1), nullptr)) atomicOr(a.ws.status, ESPO_DEV_TIMEOUT);
+    if (PADDED && all_pad[stage]) {
+      // the whole chunk is padding (nothing was copied): every token cuts the recursion with a TD error of 0, so the
+      // threads only clear their words, keep the rendezvous in step and go on to write zeros
+      fwbuf[stage * kAdvThreads + tid] = 0u;
+      pwbuf[stage * kAdvThreads + tid] = 0u;
+      if (!RET) mbar_arrive(&empty[stage]);
+      last_mask = pad_mask = (1u << kAdvPerThread) - 1u;
+#pragma unroll
+      for (int e = 0; e < kAdvPerThread; ++e) d[e] = 0.0;
+      m = Map{0.0, 0.0};
+      after = Map{0.0, 0.0};
+      cta_rendezvous(kAdvThreads);
+      return;
+    }
     float r[kAdvPerThread], v[kAdvPerThread];
 #pragma unroll
     for (int h = 0; h < kAdvPerThread / 4; ++h) {
