@@ -68,7 +68,7 @@ __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// Bulk asynchronous copy global -> shared (TMA, no tensor map, no multicast).  Both addresses
+// Bulk asynchronous copy global -> shared (TMA without a tensor map, into this CTA only).  Both addresses
 // 16-byte aligned, bytes a multiple of 16.  Completion is signalled on `bar` as transaction bytes.
 __device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
   asm volatile(
