@@ -90,3 +90,19 @@ def test_argument_errors_of_the_sharded_calls():
                              torch.empty(4, dtype=torch.uint8, device="cuda"))
     assert e.value.code == espo.ESPO_ERR_BAD_PARAM
     espo.espo_free_state(st)
+
+
+def test_sharded_step_with_row_ids_and_a_partial_batch():
+    # 7 of 12 slots take part, in scrambled order; the sharded route must treat slots exactly like espo_step does
+    cap, V = 12, 9000
+    ids = torch.tensor([9, 2, 11, 0, 5, 7, 3], dtype=torch.int32, device="cuda")
+    p = espo.make_params(temperature=1.1, mu_g=2.0, sigma2_g=4.0, beta=1.0, eps=0.1, t_max=50, sampler=espo.ESPO_SAMPLER_FLAT)
+    run = ParityRun(cap, V, p, seed=31)
+    run.launch = _sharded_launch(shard.vocab_shards(V, 3))
+    for t in range(5):
+        x = synth.logits_batch(ids.numel(), V, dtype=torch.float32, sd=2.0, seed=60 + t)
+        run.step(x, torch.rand(ids.numel(), device="cuda"), row_ids=ids)
+    view = espo.espo_state_view(run.state)
+    untouched = [s for s in range(cap) if s not in set(ids.cpu().tolist())]
+    assert torch.all(view["t"][untouched] == 0) and run.stats.row_steps >= 20
+    run.close()
