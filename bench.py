@@ -338,6 +338,36 @@ def main():
                          "traffic": None, "bytes_per_token": 12},
         }
         ADV_TOKENS_NOMINAL = n_tok
+        if not args.no_sweep:
+            # ---- the other entry points of the advantage pass on the same batch ----
+            def adv_us(fn, reps=30):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) * 1e3 / reps
+            ret = torch.empty_like(r)
+            sums = torch.zeros(2, dtype=torch.float64, device=dev)
+            t_pad = int(L.max().item())
+            pad_r = torch.zeros(ADV_B, t_pad, device=dev)
+            pad_v = torch.zeros(ADV_B, t_pad, device=dev)
+            keep = torch.arange(t_pad, device=dev)[None, :] < L[:, None]
+            pad_r[keep] = r
+            pad_v[keep] = v
+            pad_out = torch.empty_like(pad_r)
+            out["advantage_variants"] = {
+                "lambda_1_us": adv_us(lambda: espo.espo_advantages(r, v, L, s, 1.0, 1.0, -1.0, a_out)),
+                "with_returns_us": adv_us(lambda: espo.espo_advantages_returns(r, v, L, s, 1.0, 0.95, -1.0, a_out, ret)),
+                "with_batch_sums_us": adv_us(lambda: espo.espo_advantages_stats(r, v, L, s, 1.0, 0.95, -1.0, a_out, sums)),
+                "padded_layout_us": adv_us(lambda: espo.espo_advantages_padded(pad_r, pad_v, L, s, 1.0, 0.95, -1.0, pad_out)),
+                "note": f"same batch as advantage_pass; padded: [{ADV_B}, {t_pad}] ({ADV_B * t_pad} entries, {n_tok} of them tokens)",
+            }
+            del ret, pad_r, pad_v, pad_out, keep
         del r, v, L, s, a_out
 
         # ---- library operations that move the same number of bytes, timed the same way: at these sizes (one launch
