@@ -204,6 +204,18 @@ int espo_end_batch(espo_state* st, float alpha_ema, float eta_beta, float tau, f
                    float beta_max, int32_t first_update, espo_params* params_inout,
                    double* stats_out, void* stream);
 
+/* The batch boundary when the rollout batch's trajectories are spread over several states (one per GPU): every
+ * part calls espo_end_batch on a scratch copy of the parameters to obtain its stats_out, the parts exchange those six
+ * numbers (one all-gather), and every part calls this with all of them and with the real parameters.  The pooled mean,
+ * population variance and stop rate are what espo_end_batch would have found over all trajectories at once, and the
+ * same updates (Eq. 7, 8, 12) are applied to *params_inout, so all parts end with identical parameters.  Host only.
+ *   stats      host double [n_parts][6], each row as written by espo_end_batch
+ *   stats_out  host double [6] or NULL: the pooled mean, variance, rho, tokens, trajectories, stopped
+ * Errors: NULL, BAD_SHAPE, BAD_PARAM (as espo_end_batch; also negative counts or NaN in stats). */
+int espo_end_batch_merge(const double* stats, int32_t n_parts, float alpha_ema, float eta_beta, float tau,
+                         float beta_min, float beta_max, int32_t first_update, espo_params* params_inout,
+                         double* stats_out);
+
 /* ---- vocabulary shards (a tensor-parallel LM head leaves every GPU with V/N of each logit row) ----
  * The paper samples from whole rows (Algorithm 1); this pair of calls computes the same step when a row's logits
  * are spread over several buffers.  Every shard reduces its part of the rows to one espo_partial per row

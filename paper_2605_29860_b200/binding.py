@@ -79,6 +79,7 @@ def lib():
         L.espo_compact_active.argtypes = [vp, vp, vp, vp]
         L.espo_state_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.espo_end_batch.argtypes = [vp, f32, f32, f32, f32, f32, i32, C.POINTER(espo_params), C.POINTER(C.c_double), vp]
+        L.espo_end_batch_merge.argtypes = [C.POINTER(C.c_double), i32, f32, f32, f32, f32, f32, i32, C.POINTER(espo_params), C.POINTER(C.c_double)]
         L.espo_advantages.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp]
         L.espo_advantages_returns.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp]
         L.espo_advantages_stats.argtypes = [vp, vp, vp, vp, i32, i64, f32, f32, f32, vp, vp, vp, vp]
@@ -91,7 +92,7 @@ def lib():
         L.espo_last_cuda_error.argtypes = []
         for n in ("espo_init_state", "espo_reset_state", "espo_set_launch_config", "espo_step", "espo_step_partial",
                   "espo_step_merge", "espo_state_view",
-                  "espo_compact_active", "espo_state_status", "espo_end_batch", "espo_advantages", "espo_advantages_reserve",
+                  "espo_compact_active", "espo_state_status", "espo_end_batch", "espo_end_batch_merge", "espo_advantages", "espo_advantages_reserve",
                   "espo_advantages_status", "espo_advantages_noalloc", "espo_advantages_returns", "espo_advantages_stats", "espo_advantages_padded",
                   "espo_last_cuda_error"):
             getattr(L, n).restype = C.c_int
@@ -271,6 +272,24 @@ def espo_end_batch(state: EspoState, params: espo_params, alpha_ema: float = 0.9
     out = (C.c_double * 6)()
     _check(lib().espo_end_batch(state.handle, alpha_ema, eta_beta, tau, beta_min, beta_max, int(bool(first_update)),
                                 C.byref(params), out, _stream(stream)), "espo_end_batch")
+    return {"mean_g": out[0], "var_g": out[1], "stop_rate": out[2], "tokens": int(out[3]), "trajectories": int(out[4]),
+            "stopped": int(round(out[5]))}
+
+
+STATS_KEYS = ("mean_g", "var_g", "stop_rate", "tokens", "trajectories", "stopped")
+
+
+def espo_end_batch_merge(parts, params: espo_params, alpha_ema: float = 0.99, eta_beta: float = 0.1, tau: float = 0.25,
+                         beta_min: float = 0.0, beta_max: float = 3.0e38, first_update: bool = False) -> dict:
+    """Batch-boundary update from the statistics of several parts of one rollout batch (one per GPU): ``parts`` is a
+    sequence of the dicts ``espo_end_batch`` returns (or of 6-number rows in that order); see ``espo.h``.  Host only."""
+    rows = [[float(p[k]) for k in STATS_KEYS] if isinstance(p, dict) else [float(x) for x in p] for p in parts]
+    if any(len(r) != 6 for r in rows):
+        raise ValueError("every part needs six numbers: mean, variance, stop rate, tokens, trajectories, stopped")
+    flat = (C.c_double * (6 * len(rows)))(*[x for r in rows for x in r])
+    out = (C.c_double * 6)()
+    _check(lib().espo_end_batch_merge(flat, len(rows), alpha_ema, eta_beta, tau, beta_min, beta_max, int(bool(first_update)),
+                                      C.byref(params), out), "espo_end_batch_merge")
     return {"mean_g": out[0], "var_g": out[1], "stop_rate": out[2], "tokens": int(out[3]), "trajectories": int(out[4]),
             "stopped": int(round(out[5]))}
 

@@ -1747,6 +1747,46 @@ int espo_step_merge(const espo_partial* partials, int32_t n_shards, int64_t shar
   return ESPO_OK;
 }
 
+int espo_end_batch_merge(const double* stats, int32_t n_parts, float alpha_ema, float eta_beta, float tau, float beta_min,
+                         float beta_max, int32_t first_update, espo_params* params_inout, double* stats_out) {
+  if (!stats || !params_inout) return ESPO_ERR_NULL;
+  if (n_parts < 1) return ESPO_ERR_BAD_SHAPE;
+  if (!(alpha_ema >= 0.f && alpha_ema <= 1.f) || isnan(eta_beta) || isnan(tau) || isnan(beta_min) || isnan(beta_max) ||
+      beta_min > beta_max || isnan(params_inout->mu_g) || isnan(params_inout->sigma2_g) || isnan(params_inout->beta))
+    return ESPO_ERR_BAD_PARAM;
+  // pooled first and second moments of g over all parts, from each part's mean, variance and token count
+  double n = 0.0, s1 = 0.0, s2 = 0.0, traj = 0.0, stopped = 0.0;
+  for (int i = 0; i < n_parts; ++i) {
+    const double* p = stats + 6 * (size_t)i;
+    if (!(p[3] >= 0.0) || !(p[4] >= 0.0) || !(p[5] >= 0.0) || isnan(p[0]) || isnan(p[1])) return ESPO_ERR_BAD_PARAM;
+    n += p[3];
+    s1 += p[3] * p[0];
+    s2 += p[3] * (p[1] + p[0] * p[0]);
+    traj += p[4];
+    stopped += p[5];
+  }
+  double mean = 0.0, var = 0.0, rho = 0.0;
+  if (n > 0.0) {
+    mean = s1 / n;
+    var = fmax(s2 / n - mean * mean, 0.0);
+    rho = traj > 0.0 ? stopped / traj : 0.0;
+    double mu = params_inout->mu_g, sg = params_inout->sigma2_g, beta = params_inout->beta;
+    if (first_update) { mu = mean; sg = var; }
+    else {
+      mu = (double)alpha_ema * mu + (1.0 - (double)alpha_ema) * mean;        // Eq. 7
+      sg = (double)alpha_ema * sg + (1.0 - (double)alpha_ema) * var;         // Eq. 8
+    }
+    beta = fmin(fmax(beta + (double)eta_beta * (rho - (double)tau), (double)beta_min), (double)beta_max);   // Eq. 12
+    params_inout->mu_g = (float)mu;
+    params_inout->sigma2_g = (float)sg;
+    params_inout->beta = (float)beta;
+  }
+  if (stats_out) {
+    stats_out[0] = mean; stats_out[1] = var; stats_out[2] = rho; stats_out[3] = n; stats_out[4] = traj; stats_out[5] = stopped;
+  }
+  return ESPO_OK;
+}
+
 int espo_state_view(espo_state* st, const float** z, const float** g, const float** g_tilde, const float** logp,
                     const int32_t** t, const uint8_t** status, const int32_t** t_stop, const double** sum_g,
                     const double** sum_g2, const float** entropy, const double** sum_h) {

@@ -77,3 +77,18 @@ def all_gather_partials(local: torch.Tensor, dist=None) -> torch.Tensor:
     out = torch.empty((world,) + tuple(local.shape), dtype=local.dtype, device=local.device)
     dist.all_gather(list(out.unbind(0)), local.contiguous())
     return out
+
+
+def all_gather_batch_stats(stats, dist=None, device="cpu") -> list:
+    """Every rank's six batch statistics (the numbers espo_end_batch returns: mean, variance, stop rate, tokens,
+    trajectories, stopped), in rank order -- the input of espo_end_batch_merge.  The only collective the row-sharded
+    method needs, once per training batch."""
+    row = [float(x) for x in stats]
+    if len(row) != 6:
+        raise ValueError("six numbers per rank")
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return [row]
+    mine = torch.tensor(row, dtype=torch.float64, device=device)
+    out = [torch.empty_like(mine) for _ in range(dist.get_world_size())]
+    dist.all_gather(out, mine)
+    return [t.tolist() for t in out]

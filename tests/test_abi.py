@@ -61,3 +61,31 @@ def test_python_binding_mirrors_the_abi():
             continue
         assert hasattr(espo, name), f"binding lacks {name}"
     assert ctypes.sizeof(espo.espo_params) == 76
+
+
+def test_end_batch_merge_pools_the_parts_statistics(lib):
+    # host-only entry point: pooled mean / population variance / stop rate of parts given by (mean, var, rho, n, traj, stopped)
+    import numpy as np
+    import paper_2605_29860_b200 as espo
+    rng = np.random.default_rng(0)
+    groups = [rng.gamma(2.0, 1.5, size=n) for n in (1200, 1, 35000)]
+    traj, stopped = [40, 1, 300], [10, 0, 77]
+    parts = [[g.mean(), g.var(), s / t, g.size, t, s] for g, t, s in zip(groups, traj, stopped)] + [[0.0, 0.0, 0.0, 0, 0, 0]]
+    allg = np.concatenate(groups)
+    for first in (False, True):
+        p = espo.make_params(mu_g=2.0, sigma2_g=3.0, beta=7.0)
+        st = espo.espo_end_batch_merge(parts, p, alpha_ema=0.9, eta_beta=0.5, tau=0.25, beta_min=0.0, beta_max=7.05,
+                                       first_update=first)
+        rho = sum(stopped) / sum(traj)
+        assert abs(st["mean_g"] - allg.mean()) < 1e-12 and abs(st["var_g"] - allg.var()) < 1e-10 and abs(st["stop_rate"] - rho) < 1e-15
+        assert (st["tokens"], st["trajectories"], st["stopped"]) == (allg.size, sum(traj), sum(stopped))
+        want_mu = allg.mean() if first else 0.9 * 2.0 + 0.1 * allg.mean()              # Eq. 7
+        want_s2 = allg.var() if first else 0.9 * 3.0 + 0.1 * allg.var()                # Eq. 8
+        want_beta = min(max(7.0 + 0.5 * (rho - 0.25), 0.0), 7.05)                      # Eq. 12, clipped
+        assert abs(p.mu_g - want_mu) < 1e-6 and abs(p.sigma2_g - want_s2) < 1e-6 and abs(p.beta - want_beta) < 1e-6
+    q = espo.make_params(mu_g=2.0, sigma2_g=3.0, beta=7.0)
+    espo.espo_end_batch_merge([[0.0] * 6], q)                                          # no tokens: nothing changes
+    assert (q.mu_g, q.sigma2_g, q.beta) == (2.0, 3.0, 7.0)
+    import pytest
+    with pytest.raises(espo.EspoError):
+        espo.espo_end_batch_merge([[1.0, 1.0, 0.0, -5, 1, 0]], q)

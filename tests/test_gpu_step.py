@@ -320,6 +320,34 @@ def test_end_batch_updates_statistics_and_beta_like_the_oracle():
     run.close()
 
 
+def test_end_batch_over_two_states_equals_the_oracle_over_all_trajectories():
+    # the rollout batch split over two states (as over two GPUs); each gives its six statistics, the merge pools them
+    V, T = 5000, 8
+    p = espo.make_params(temperature=1.0, mu_g=0.5, sigma2_g=1.0, alpha_s=0.6, beta=1.0, eps=0.2)
+    whole = oracle.Rollout(50, seed=0)               # stands for all trajectories; slots 0..29 and 30..49
+    parts = []
+    for lo, n, seed in ((0, 30, 41), (30, 20, 42)):
+        run = ParityRun(n, V, p, seed=seed)
+        for t in range(T):
+            x = synth.logits_batch(n, V, dtype=torch.bfloat16, sd=2.5, seed=800 + 10 * lo + t)
+            run.step(x, torch.rand(n, device="cuda", generator=torch.Generator("cuda").manual_seed(lo + t)))
+        assert not run.dropped
+        for s_ in range(n):
+            whole.states[lo + s_] = run.ro.states[s_]
+        scratch = espo.make_params(mu_g=2.0, sigma2_g=3.0, beta=7.0)
+        parts.append(espo.espo_end_batch(run.state, scratch, alpha_ema=0.9, eta_beta=0.5, tau=0.25, beta_max=7.2))
+        run.close()
+    for first in (False, True):
+        q = espo.make_params(mu_g=2.0, sigma2_g=3.0, beta=7.0)
+        st = espo.espo_end_batch_merge(parts, q, alpha_ema=0.9, eta_beta=0.5, tau=0.25, beta_min=0.0, beta_max=7.2,
+                                       first_update=first)
+        mu, s2, beta, ost = whole.end_batch(2.0, 3.0, 7.0, alpha_ema=0.9, eta_beta=0.5, tau=0.25, beta_min=0.0,
+                                            beta_max=7.2, first_update=first)
+        assert close(q.mu_g, mu) and close(q.sigma2_g, s2) and close(q.beta, beta)
+        assert close(st["mean_g"], ost[0]) and close(st["var_g"], ost[1]) and close(st["stop_rate"], ost[2])
+        assert (st["tokens"], st["trajectories"], st["stopped"]) == (int(ost[3]), 50, int(ost[5]))
+
+
 def test_reset_state_starts_a_new_batch():
     B, V = 4, 4096
     p = espo.make_params(mu_g=1.0, sigma2_g=2.0, beta=100.0)

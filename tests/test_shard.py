@@ -38,7 +38,8 @@ def _worker(rank, world, port, out_dir):
     # vocabulary shards: each rank contributes its partials, everyone ends with [world, rows, 8] in rank order
     mine = torch.full((5, 8), float(rank + 1)) + torch.arange(5, dtype=torch.float32)[:, None]
     gathered = shard.all_gather_partials(mine, dist)
-    torch.save({"ms": ms, "tot": tot, "seeds": seeds, "plan": plan, "gathered": gathered}, os.path.join(out_dir, f"r{rank}.pt"))
+    stats = shard.all_gather_batch_stats([1.0 + rank, 0.5, 0.25, 100 * (rank + 1), 10, 2 + rank], dist)
+    torch.save({"ms": ms, "tot": tot, "seeds": seeds, "plan": plan, "gathered": gathered, "stats": stats}, os.path.join(out_dir, f"r{rank}.pt"))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -51,6 +52,7 @@ def test_two_ranks_shard_rows_and_reduce_timings(tmp_path):
         assert r["ms"] == [11.0, 5.0]                    # max over ranks, element-wise, same on every rank
         assert r["tot"] == [1024.0, 1.0]
         assert r["plan"]["global_rows"] == 1024
+        assert r["stats"] == [[1.0, 0.5, 0.25, 100.0, 10.0, 2.0], [2.0, 0.5, 0.25, 200.0, 10.0, 3.0]]
         g = r["gathered"]
         assert tuple(g.shape) == (world, 5, 8) and g.is_contiguous()
         for k in range(world):
