@@ -126,26 +126,6 @@ __global__ void __launch_bounds__(kPrepThreads) espo_adv_prep_kernel(const AdvAr
   if (bad) atomicOr(a.ws.status, ESPO_DEV_BAD_LENGTHS);
 }
 
-// Preparation for the padded layout [B, t_max]: row i starts at token i*t_max, so offsets and chunk owners are
-// plain arithmetic; lengths outside [0, t_max] are reported (the scan clamps them).
-__global__ void __launch_bounds__(kPrepThreads) espo_adv_prep_padded_kernel(const AdvArgs a) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  bool bad = false;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i <= a.B; i += stride) {
-    a.ws.offsets[i] = i * a.t_max;
-    if (i < a.B) {
-      const int len = a.lengths[i];
-      bad |= (len < 0 || len > a.t_max);
-    }
-  }
-  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < a.nchunks; j += stride) {
-    const long long i = j * kAdvChunk / a.t_max;
-    a.ws.chunk_first[j] = (int)(i < a.B ? i : a.B - 1);
-  }
-  if (bad) atomicOr(a.ws.status, ESPO_DEV_BAD_LENGTHS);
-}
-
 // ---------------------------------------------------------------------------------------
 // The scan.
 // ---------------------------------------------------------------------------------------
@@ -290,11 +270,13 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     // the preparation flags) are pulled into range.
     auto cand_lo = [&](int k) -> int {
       const long long p0 = t_hi - (long long)(k + 1) * kAdvChunk;
+      if (PADDED) return (int)min(max(p0, t_lo) / a.t_max, (long long)a.B);      // rows are t_max apart: no table needed
       const int c = __ldcg(a.ws.chunk_first + (max(p0, t_lo) / kAdvChunk));
       return c < 0 ? 0 : (c > a.B ? a.B : c);
     };
     auto cand_hi = [&](int k) -> int {
       const long long p_end = min(t_hi - (long long)k * kAdvChunk, a.total);
+      if (PADDED) return (int)min((p_end - 1) / a.t_max, (long long)a.B - 1);
       const long long g = (p_end - 1) / kAdvChunk + 1;
       if (g >= a.nchunks) return a.B - 1;
       const int c = __ldcg(a.ws.chunk_first + g);
@@ -354,7 +336,7 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     const int pre = nck < kAdvStages ? nck : kAdvStages;
     if (lane == 0)
       for (int k = 0; k < pre; ++k) issue_copies(k);       // needs nothing of the preparation kernel
-    asm volatile("griddepcontrol.wait;" ::: "memory");     // everything below reads what it wrote
+    if (!PADDED) asm volatile("griddepcontrol.wait;" ::: "memory");     // everything below reads what the preparation wrote
     int c_lo = cand_lo(0), c_hi = cand_hi(0);               // candidates of the chunk in hand
     int n_lo = nck > 1 ? cand_lo(1) : 0, n_hi = nck > 1 ? cand_hi(1) : -1;   // and of the next one
     Traj t0 = traj_load(c_lo + lane, c_hi);                 // the lane's first candidate, loaded one chunk ahead
@@ -474,14 +456,19 @@ __global__ void __launch_bounds__(kAdvCtaThreads, kAdvCtasPerSm) espo_adv_scan_k
     for (int w = warp + 1; w < kAdvWarps; ++w) after = compose(after, warp_agg[par][w]);
   };
 
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // everything below reads what the preparation kernel wrote
+  if (!PADDED) asm volatile("griddepcontrol.wait;" ::: "memory");   // everything below reads what the preparation kernel wrote
+  if (PADDED && blockIdx.x == 0) {   // no preparation kernel looked at the lengths
+    bool bad = false;
+    for (int i = tid; i < a.B; i += kAdvThreads) { const int len = a.lengths[i]; bad |= (len < 0 || len > a.t_max); }
+    if (bad) atomicOr(a.ws.status, ESPO_DEV_BAD_LENGTHS);
+  }
 
   // ---- the advantage of the token that follows the range (token t_hi).  Its trajectory continues in the next CTA's
   //      range; unrolled, Eq. 5 makes it the weighted sum of the rest of that one trajectory's TD errors,
   //      sum_k (gamma*lambda)^k delta_k, which the CTA's threads take straight from global memory (read only, usually
   //      served by L2): thread t owns tokens 4t .. 4t+3 of every 1024.  CTAs therefore never wait for one another. ----
   if (nck > 0 && t_hi < a.total) {   // find the trajectory that holds token t_hi
-    int first = __ldcg(a.ws.chunk_first + (t_hi / kAdvChunk));
+    int first = PADDED ? (int)min(t_hi / a.t_max, (long long)a.B) : __ldcg(a.ws.chunk_first + (t_hi / kAdvChunk));
     if ((unsigned)first >= (unsigned)a.B) first = a.B;   // only with inconsistent lengths (flagged by the preparation)
     for (int i = first + tid; i < a.B; i += kAdvThreads) {
       long long o0, o1;
@@ -694,9 +681,12 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
       ESPO_CUDA_TRY(cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAdvSmemBytes));
     attr_set[dev] = true;
   }
-  if (a.t_max > 0) espo_adv_prep_padded_kernel<<<8, kPrepThreads, 0, s>>>(a);
-  else espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
-  ESPO_CUDA_TRY(cudaGetLastError());
+  // The packed layout needs offsets and chunk owners from a preparation kernel, and the scan is launched as its
+  // programmatic dependent so that its ring fills meanwhile; the padded layout's offsets are arithmetic: one launch.
+  if (a.t_max == 0) {
+    espo_adv_prep_kernel<<<1, kPrepThreads, 0, s>>>(a);
+    ESPO_CUDA_TRY(cudaGetLastError());
+  }
   long long grid = (long long)sm_count * kAdvCtasPerSm;
   if (grid > a.nchunks) grid = a.nchunks;
   cudaLaunchConfig_t cfg = {};
@@ -707,8 +697,10 @@ static int launch_advantages(const AdvArgs& a, int sm_count, cudaStream_t s) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start before the preparation kernel ends
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  if (a.t_max == 0) {
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
   if (a.t_max > 0 && a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, true, true>, a));
   else if (a.t_max > 0) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<false, false, true>, a));
   else if (a.stats && a.ret) ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo_adv_scan_kernel<true, true, false>, a));
