@@ -220,6 +220,9 @@ __device__ __forceinline__ void reduce_block(const StepArgs& a, const unsigned c
       if (j & 1) acc1 = __fadd2_rn(acc1, e); else acc0 = __fadd2_rn(acc0, e);
     }
   }
+  // (The exponents were x*k2 + c0 with c0 = -ref*k2 rounded once, so every one of them is off by the same
+  // dlt = c0 + ref*k2, the rounding error of that product: up to 1e-5 at low temperatures.  The warp that reads the
+  // record takes the common factor 2^dlt out again; see finalize_row.)
   const float s_b = warp_sum((acc0.x + acc0.y) + (acc1.x + acc1.y));
 
   if (SAMPLER == ESPO_SAMPLER_FLAT) {
@@ -305,7 +308,8 @@ __device__ __forceinline__ float sum_exp2_32(const float (&x)[kSubIds], float m,
     const float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
     if (i & 1) acc1 = __fadd2_rn(acc1, e); else acc0 = __fadd2_rn(acc0, e);
   }
-  return (acc0.x + acc0.y) + (acc1.x + acc1.y);
+  // every exponent is off by the rounding error of m*k2 (see reduce_block): one factor takes it out
+  return ((acc0.x + acc0.y) + (acc1.x + acc1.y)) * ex2_approx(-fmaf(m, k2, c0));
 }
 
 // What one thread does once a row's token is known: regret, normalisation, smoothing, stop rule and bookkeeping
@@ -414,6 +418,18 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
       const int b = base + 32 * i + lane;
       // shared-memory table or global records written by other CTAs: one generic load that bypasses L1 serves both
       r[i] = (b < a.nblk) ? ld_volatile_f4(static_cast<const float4*>(rec_row) + b) : make_float4(NINF, 0.f, NINF, __int_as_float(-1));
+    }
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+      // The block's exponents were all off by dlt = fl(-m_b*k2) + m_b*k2 (reduce_block), which the fused
+      // multiply-add returns exactly: s_b and u_b carry a factor 2^dlt (and u_b the shift dlt*s_b); to first
+      // order in dlt <= 1e-4 that is taken out here.
+      const float dlt = fmaf(r[i].x, a.k2, -r[i].x * a.k2);
+      if (r[i].y > 0.f && !isinf(r[i].y)) {
+        const float s_c = fmaf(r[i].y, -0.6931471805599453f * dlt, r[i].y);
+        if (SAMPLER == ESPO_SAMPLER_HIER) r[i].z = fmaf(r[i].z, -0.6931471805599453f * dlt, r[i].z) - dlt * s_c;
+        r[i].y = s_c;
+      }
     }
     float lm = run_m;
 #pragma unroll
@@ -1191,9 +1207,8 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
       for (int j = 1; j < VEC; ++j) vm = fmaxf(vm, x[j]);
       if (vm > m) { s_t *= ex2_approx((m - vm) * a.k2); m = vm; }   // m = -inf: s_t is 0 and stays 0
       if (m > NINF) {
-        const float c0 = -m * a.k2;
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) s_t += ex2_approx(fmaf(x[j], a.k2, c0));   // NaN stays NaN; +inf makes m +inf, then NaN
+        for (int j = 0; j < VEC; ++j) s_t += ex2_approx((x[j] - m) * a.k2);     // NaN stays NaN; +inf makes m +inf, then NaN
       } else {
 #pragma unroll
         for (int j = 0; j < VEC; ++j) if (x[j] != x[j]) s_t = x[j];             // a NaN among logits that are all -inf so far

@@ -291,6 +291,23 @@ def test_policy_entropy_in_the_same_pass(V, dtype, temperature):
     run.close()
 
 
+@pytest.mark.parametrize("sampler", SAMPLERS)
+@pytest.mark.parametrize("temperature", [0.05, 0.2, 3.0, 10.0])
+def test_temperatures_far_from_one(temperature, sampler):
+    # At T = 0.05 a logit is scaled by 20/ln 2 before the exponential, so the rounding of that scale times a block's
+    # maximum is of the order 1e-5 in log pi unless the kernel takes it out; at T = 10 the row is nearly flat.
+    B, T = 12, 3
+    for V, dtype in ((152064, torch.bfloat16), (32000, torch.float32), (1000, torch.bfloat16)):
+        p = espo.make_params(temperature=temperature, mu_g=1.0, sigma2_g=4.0, beta=2.0, eps=0.1, t_max=6,
+                             sampler=sampler, want_entropy=int(sampler == espo.ESPO_SAMPLER_HIER))
+        run = ParityRun(B, V, p, seed=int(temperature * 100) + V)
+        for t in range(T):
+            run.step(synth.logits_batch(B, V, dtype=dtype, sd=3.0, seed=t + int(temperature * 10)),
+                     torch.rand(B, device="cuda", generator=torch.Generator("cuda").manual_seed(V + t)))
+        assert run.stats.token_ties <= 2, (V, run.stats)
+        run.close()
+
+
 def sum_h_of(run, slot):
     return float(sum(run.entropy_log[slot]))
 
