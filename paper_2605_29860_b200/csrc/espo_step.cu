@@ -422,12 +422,14 @@ __device__ __noinline__ void finalize_row(const StepArgs& a, int row, int lane, 
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i) {
       // The block's exponents were all off by dlt = fl(-m_b*k2) + m_b*k2 (reduce_block), which the fused
-      // multiply-add returns exactly: s_b and u_b carry a factor 2^dlt (and u_b the shift dlt*s_b); to first
-      // order in dlt <= 1e-4 that is taken out here.
+      // multiply-add returns exactly: s_b and u_b carry a factor 2^dlt (and u_b the shift dlt*s_b), taken out here.
+      // dlt is half an ulp of m_b*k2 at most: 1e-5 for logits of some tens at low temperature, more for rows that
+      // sit at a large offset.
       const float dlt = fmaf(r[i].x, a.k2, -r[i].x * a.k2);
       if (r[i].y > 0.f && !isinf(r[i].y)) {
-        const float s_c = fmaf(r[i].y, -0.6931471805599453f * dlt, r[i].y);
-        if (SAMPLER == ESPO_SAMPLER_HIER) r[i].z = fmaf(r[i].z, -0.6931471805599453f * dlt, r[i].z) - dlt * s_c;
+        const float f = ex2_approx(-dlt);
+        const float s_c = r[i].y * f;
+        if (SAMPLER == ESPO_SAMPLER_HIER) r[i].z = fmaf(r[i].z, f, -dlt * s_c);
         r[i].y = s_c;
       }
     }

@@ -308,6 +308,23 @@ def test_temperatures_far_from_one(temperature, sampler):
         run.close()
 
 
+@pytest.mark.parametrize("sampler", SAMPLERS)
+@pytest.mark.parametrize("offset,scale", [(1000.0, 1.0), (-5000.0, 1.0), (30000.0, 1.0), (200.0, 10.0)])
+def test_rows_at_a_large_offset_or_scale(offset, scale, sampler):
+    # log-softmax does not change when a row is shifted; the kernel's scaled exponent offsets must not either
+    B = 8
+    for V, dtype in ((152064, torch.float32), (5000, torch.bfloat16)):
+        p = espo.make_params(temperature=0.3, mu_g=1.0, sigma2_g=4.0, beta=2.0, eps=0.1, t_max=6, sampler=sampler,
+                             want_entropy=int(sampler == espo.ESPO_SAMPLER_HIER))
+        run = ParityRun(B, V, p, seed=V)
+        for t in range(2):
+            x = synth.logits_batch(B, V, dtype=torch.float32, sd=3.0, seed=t + 3)
+            run.step((x * scale + offset).to(dtype),
+                     torch.rand(B, device="cuda", generator=torch.Generator("cuda").manual_seed(t)))
+        assert run.stats.token_ties <= 2, (V, run.stats)
+        run.close()
+
+
 def sum_h_of(run, slot):
     return float(sum(run.entropy_log[slot]))
 
