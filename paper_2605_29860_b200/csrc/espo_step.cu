@@ -988,9 +988,12 @@ constexpr int kFiltThreads = 1024;
 constexpr int kFiltWarps = kFiltThreads / 32;
 constexpr int kFiltSeg = 320;                      // candidate-list entries per warp
 constexpr int kFiltCopies = 16;                    // private copies of the digit histogram (two warps share one)
-constexpr size_t kFiltSmemBytes = (size_t)kFiltCopies * 256 * sizeof(uint4) +
+constexpr int kFiltRing = 4;                       // 16-byte pieces a thread keeps in flight during the pass over the row
+constexpr size_t kFiltRingBytes = (size_t)kFiltRing * kFiltThreads * 16;
+static_assert(kFiltRingBytes >= (size_t)kFiltCopies * 256 * sizeof(uint4), "the histograms reuse the ring's memory");
+constexpr size_t kFiltSmemBytes = kFiltRingBytes +
                                   256 * (sizeof(unsigned long long) + sizeof(unsigned)) + 192 * sizeof(float) +
-                                  (size_t)kFiltWarps * kFiltSeg * sizeof(uint2) + 128;
+                                  (size_t)kFiltWarps * kFiltSeg * (sizeof(uint2) + sizeof(unsigned)) + 128;
 
 // A probability mass e in [0, 1] as an integer count of 2^-40 (exact for a float; two 32-bit conversions).
 __device__ __forceinline__ unsigned long long filt_fixed(float e) {
@@ -1063,18 +1066,20 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
   // digit histograms: per bin the mass as three limbs of 14 + 13 + 13 bits (32-bit shared-memory atomics are native,
   // 64-bit ones are not; a copy sees fewer than 2^18 logits per pass, so no limb overflows) and the count
   uint4* whist = reinterpret_cast<uint4*>(fsm);                                          // [copies][256]
-  unsigned long long* bmass = reinterpret_cast<unsigned long long*>(whist + kFiltCopies * 256);   // [256] all copies together
+  unsigned char* ring = fsm;                             // the row pass's landing slots (the histograms are idle then)
+  unsigned long long* bmass = reinterpret_cast<unsigned long long*>(fsm + kFiltRingBytes);   // [256] all copies together
   unsigned* bcnt = reinterpret_cast<unsigned*>(bmass + 256);                             // [256]
   float* red_f = reinterpret_cast<float*>(bcnt + 256);                                   // [32] scores / sums
   int* red_i = reinterpret_cast<int*>(red_f + 32);                                       // [32] ids, flags
   unsigned long long* red_u = reinterpret_cast<unsigned long long*>(red_i + 32);         // [2][32] integer sums
   uint2* cand = reinterpret_cast<uint2*>(red_u + 64);                                    // [warps][kFiltSeg] (id, bits)
+  unsigned* glist = reinterpret_cast<unsigned*>(cand + kFiltWarps * kFiltSeg);           // [warps][kFiltSeg] first ids of groups with a candidate
   unsigned* sbin = reinterpret_cast<unsigned*>(whist);                                   // 4096 sample bins (before the digit passes)
   __shared__ RowPre pre_s;
   __shared__ unsigned long long sh_acc_mass, sh_kept_mass;
   __shared__ unsigned sh_acc_cnt, sh_prefix, sh_cut_a;
   __shared__ int sh_found, sh_overflow;
-  __shared__ unsigned seg_n[kFiltWarps];
+  __shared__ unsigned seg_n[kFiltWarps], seg_g[kFiltWarps];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float NINF = __int_as_float(0xff800000);
@@ -1083,7 +1088,7 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
   for (int row = blockIdx.x; row < a.n_rows; row += gridDim.x) {
     __syncthreads();                                         // the previous row's shared values are no longer read
     if (tid == 0) { pre_s = prefetch_row(a, row); sh_overflow = 0; sh_cut_a = 0u; }
-    if (tid < kFiltWarps) seg_n[tid] = 0u;
+    if (tid < kFiltWarps) { seg_n[tid] = 0u; seg_g[tid] = 0u; }
     for (int i = tid; i < 4096; i += kFiltThreads) sbin[i] = 0u;
     __syncthreads();
     const RowPre pre = pre_s;
@@ -1122,33 +1127,43 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
       }
     };
     auto value_of = [&](uint32_t bits) -> float { return __uint_as_float(ES == 2 ? bits << 16 : bits); };
-    // The two passes over the whole row work on groups of VEC consecutive logits, already as floats: fn(first id,
+    // The pass over the whole row works on groups of VEC consecutive logits, already as floats: fn(first id,
     // values); positions past the row's end read as -inf, which no pass counts.
     auto for_each_group = [&](auto&& fn) {
       const int v_main = vec_ok ? (a.V / VEC) * VEC : 0;
-      constexpr int kInFlight = 4;
-      for (int base0 = tid * VEC; base0 < v_main; base0 += kInFlight * kFiltThreads * VEC) {
-        uint4 q[kInFlight];
+      // Every thread copies its own 16-byte pieces of the row (piece number g * threads + tid) into its own slots of
+      // a ring in shared memory, kFiltRing - 1 pieces ahead of the one it works on, so that the loads of the whole
+      // CTA keep the memory pipe full while the arithmetic runs; no other thread reads the slots: no barrier.
+      const int n_vec = v_main / VEC;
+      const int n_mine = n_vec > tid ? (n_vec - tid + kFiltThreads - 1) / kFiltThreads : 0;
+      const int n_warp = __shfl_sync(kFullMask, n_mine, 0);          // lane 0 has the most pieces: the warp calls fn together
+      const uint32_t slot0 = smem_addr(ring) + (uint32_t)tid * 16u;
+      const unsigned char* src0 = row_base + (size_t)tid * 16;
+      auto issue = [&](int g) {
+        if (g < n_mine)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + (uint32_t)(g % kFiltRing) * (kFiltThreads * 16u)),
+                       "l"(src0 + (size_t)g * (kFiltThreads * 16)) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");       // one group per piece, empty past the end
+      };
+      for (int g = 0; g < kFiltRing - 1; ++g) issue(g);
+      for (int g = 0; g < n_warp; ++g) {
+        issue(g + kFiltRing - 1);                                   // into the slot read one turn ago
+        asm volatile("cp.async.wait_group %0;" ::"n"(kFiltRing - 1) : "memory");
+        uint4 q = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // -inf in either format: no piece left
+        if (ES == 4) q = make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+        if (g < n_mine) q = *reinterpret_cast<const uint4*>(ring + (size_t)(g % kFiltRing) * (kFiltThreads * 16) + (size_t)tid * 16);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+        float x[VEC];
 #pragma unroll
-        for (int u = 0; u < kInFlight; ++u) {
-          const int base = base0 + u * kFiltThreads * VEC;
-          q[u] = (base < v_main) ? __ldg(reinterpret_cast<const uint4*>(row_base + (size_t)base * ES)) : make_uint4(0u, 0u, 0u, 0u);
+        for (int j = 0; j < 4; ++j) {
+          if (ES == 2) { x[2 * j] = __uint_as_float(w[j] << 16); x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
+          else x[j] = __uint_as_float(w[j]);
         }
-#pragma unroll
-        for (int u = 0; u < kInFlight; ++u) {
-          const int base = base0 + u * kFiltThreads * VEC;
-          if (base >= v_main) break;
-          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-          float x[VEC];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (ES == 2) { x[2 * j] = __uint_as_float(w[j] << 16); x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
-            else x[j] = __uint_as_float(w[j]);
-          }
-          fn(base, x);
-        }
+        fn((g * kFiltThreads + tid) * VEC, x);
       }
-      for (int base = v_main + tid * VEC; base < a.V; base += kFiltThreads * VEC) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      for (int base_w = v_main + (tid - lane) * VEC; base_w < a.V; base_w += kFiltThreads * VEC) {   // the same trips for a warp
+        const int base = base_w + lane * VEC;
         float x[VEC];
 #pragma unroll
         for (int j = 0; j < VEC; ++j) x[j] = (base + j < a.V) ? load_logit<ES>(row_base, base + j) : NINF;
@@ -1203,6 +1218,7 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     //      turns the thread's sum into NaN or its maximum into +inf); logits at or above the cut go onto the list. ----
     float m = NINF, s_t = 0.f;
     uint2* my_seg = cand + warp * kFiltSeg;
+    unsigned* my_groups = glist + warp * kFiltSeg;
     for_each_group([&](int base, const float (&x)[VEC]) {
       float vm = x[0];
 #pragma unroll
@@ -1215,23 +1231,56 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
 #pragma unroll
         for (int j = 0; j < VEC; ++j) if (x[j] != x[j]) s_t = x[j];             // a NaN among logits that are all -inf so far
       }
+      // About one logit in 50 lies above the cut, so in nearly every trip some lane of the warp has one, and what the
+      // lane does about it the whole warp waits for: the pass only notes the group on the warp's list of groups
+      // (measured: faster than listing the logits here, and than bit masks in registers scanned afterwards).
       if (vm >= cut_x) {
+        const unsigned at = atomicAdd(&seg_g[warp], 1u);
+        if (at < (unsigned)kFiltSeg) my_groups[at] = (unsigned)base;
+        else sh_overflow = 1;
+      }
+    });
+    // ---- the noted groups, read again (L2, a few per lane), give the list of candidates ----
+    __syncwarp();
+    {
+      const unsigned n_g = min(seg_g[warp], (unsigned)kFiltSeg);
+      const int v_main = vec_ok ? (a.V / VEC) * VEC : 0;
+      for (unsigned i = lane; i < n_g; i += 32) {
+        const int base = (int)my_groups[i];
+        float x[VEC];
+        if (base + VEC <= v_main) {                          // a whole 16-byte piece of an aligned row
+          const uint4 q = __ldg(reinterpret_cast<const uint4*>(row_base + (size_t)base * ES));
+          const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (ES == 2) { x[2 * j] = __uint_as_float(w[j] << 16); x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
+            else x[j] = __uint_as_float(w[j]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) x[j] = (base + j < a.V) ? load_logit<ES>(row_base, base + j) : NINF;
+        }
+        unsigned n_c = 0u;
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) n_c += (x[j] >= cut_x) ? 1u : 0u;
+        unsigned at = atomicAdd(&seg_n[warp], n_c);
 #pragma unroll
         for (int j = 0; j < VEC; ++j) {
           if (!(x[j] >= cut_x)) continue;
-          const unsigned at = atomicAdd(&seg_n[warp], 1u);
           if (at < (unsigned)kFiltSeg) my_seg[at] = make_uint2((unsigned)(base + j), bits_of(x[j]));
           else sh_overflow = 1;
+          ++at;
         }
       }
-    });
+    }
     bool poisoned = (s_t != s_t) || (m == __int_as_float(0x7f800000));
     const float wm = warp_max(m);
     poisoned = __any_sync(kFullMask, poisoned);
     if (lane == 0) { red_f[warp] = wm; red_i[warp] = poisoned; }
     __syncthreads();
-    float M = NINF;
-    for (int w = 0; w < kFiltWarps; ++w) { M = fmaxf(M, red_f[w]); poisoned |= red_i[w] != 0; }
+    static_assert(kFiltWarps == 32, "one lane per warp's partial result");
+    const float M = warp_max(red_f[lane]);                   // every warp folds the 32 partial results by itself
+    poisoned = __any_sync(kFullMask, red_i[lane] != 0);
     if (poisoned || !(M > NINF)) { mark_row(a, row, pre.slot, tid, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true); continue; }
     float tot_f = (m > NINF) ? s_t * ex2_approx((m - M) * a.k2) : 0.f;
     tot_f = warp_sum(tot_f);                                 // fixed order: the same bits on every call
@@ -1248,9 +1297,14 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     __syncthreads();
     if (lane == 0) { red_f[warp] = tot_f; red_u[warp] = m_a; red_u[32 + warp] = c_a; }
     __syncthreads();
-    double tot = 0.0;
-    unsigned long long ma = 0ull, ca = 0ull;                 // integer sums: the order does not matter
-    for (int w = 0; w < kFiltWarps; ++w) { tot += (double)red_f[w]; ma += red_u[w]; ca += red_u[32 + w]; }
+    double tot = (double)red_f[lane];                        // butterfly: the same tree, hence the same bits, in every lane and call
+    unsigned long long ma = red_u[lane], ca = red_u[32 + lane];   // integer sums: the order does not matter
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      tot += __shfl_xor_sync(kFullMask, tot, o);
+      ma += __shfl_xor_sync(kFullMask, ma, o);
+      ca += __shfl_xor_sync(kFullMask, ca, o);
+    }
     const unsigned long long total = (unsigned long long)(tot * 1099511627776.0);
     const unsigned long long pf = (a.top_p < 1.f) ? (unsigned long long)((double)total * (double)a.top_p) : ~0ull;   // top_p of the row's mass
     const unsigned long long kf = a.top_k > 0 ? (unsigned long long)a.top_k : ~0ull;
