@@ -1087,13 +1087,13 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
 
   for (int row = blockIdx.x; row < a.n_rows; row += gridDim.x) {
     __syncthreads();                                         // the previous row's shared values are no longer read
-    if (tid == 0) { pre_s = prefetch_row(a, row); sh_overflow = 0; sh_cut_a = 0u; }
+    // Thread 0 asks for the row's state now and hands it over at the barrier after the sampling phase, so that the
+    // loads (a chain of two or three) are under way while the CTA samples the row.
+    RowPre pre_r;
+    if (tid == 0) { pre_r = prefetch_row(a, row); sh_overflow = 0; sh_cut_a = 0u; }
     if (tid < kFiltWarps) { seg_n[tid] = 0u; seg_g[tid] = 0u; }
     for (int i = tid; i < 4096; i += kFiltThreads) sbin[i] = 0u;
     __syncthreads();
-    const RowPre pre = pre_s;
-    if (pre.slot < 0) { mark_row(a, row, 0, tid, -1, ESPO_DEV_BAD_SLOT, -1, true); continue; }
-    if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, pre.slot, tid, -1, 0u, -1, true); continue; }   // finished: untouched
 
     const unsigned char* row_base = a.logits + (size_t)row * a.row_stride_bytes;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(row_base) & 15u) == 0;
@@ -1206,7 +1206,11 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
         }
       }
     }
+    if (tid == 0) pre_s = pre_r;
     __syncthreads();
+    const RowPre pre = pre_s;
+    if (pre.slot < 0) { mark_row(a, row, 0, tid, -1, ESPO_DEV_BAD_SLOT, -1, true); continue; }
+    if (pre.status != ESPO_ROW_ACTIVE) { mark_row(a, row, pre.slot, tid, -1, 0u, -1, true); continue; }   // finished: untouched
     const uint32_t cut_a = sh_cut_a;
     // the cut as a logit: keys are monotone in the value, so key >= cut_a is x >= cut_x
     const uint32_t key_top = (ES == 2) ? 0x8000u : 0x80000000u;
@@ -1400,17 +1404,18 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     __syncthreads();                                         // red_f / red_i of the sums above are no longer read
     if (lane == 0) { red_f[warp] = best; red_i[warp] = best_id; }
     __syncthreads();
-    if (tid == 0) {
-      float b = NINF;
-      int tok = -1;
-      for (int w = 0; w < kFiltWarps; ++w)
-        if (red_i[w] >= 0 && (tok < 0 || red_f[w] > b || (red_f[w] == b && red_i[w] < tok))) { b = red_f[w]; tok = red_i[w]; }
-      if (tok < 0) {
-        mark_row(a, row, pre.slot, 0, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true);
-      } else {
-        const float l_tok = load_logit<ES>(row_base, tok);
-        const float S = (float)((double)kept_mass * (1.0 / 1099511627776.0));
-        commit_row(a, row, pre, ds, M, S, logf(S), 0.f, l_tok, tok, true);
+    if (warp == 0) {
+      float b = red_f[lane];
+      int tok = red_i[lane];
+      warp_argmax(b, tok);                                   // largest score, the smaller id among equal ones, -1 if none
+      if (lane == 0) {
+        if (tok < 0) {
+          mark_row(a, row, pre.slot, 0, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true);
+        } else {
+          const float l_tok = load_logit<ES>(row_base, tok);
+          const float S = (float)((double)kept_mass * (1.0 / 1099511627776.0));
+          commit_row(a, row, pre, ds, M, S, logf(S), 0.f, l_tok, tok, true);
+        }
       }
     }
   }
