@@ -1249,31 +1249,44 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     {
       const unsigned n_g = min(seg_g[warp], (unsigned)kFiltSeg);
       const int v_main = vec_ok ? (a.V / VEC) * VEC : 0;
-      for (unsigned i = lane; i < n_g; i += 32) {
-        const int base = (int)my_groups[i];
-        float x[VEC];
-        if (base + VEC <= v_main) {                          // a whole 16-byte piece of an aligned row
-          const uint4 q = __ldg(reinterpret_cast<const uint4*>(row_base + (size_t)base * ES));
-          const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+      constexpr int kAhead = 4;                              // groups a lane asks for before it takes the first apart
+      for (unsigned i0 = lane; i0 < n_g; i0 += 32 * kAhead) {
+        int base[kAhead];
+        uint4 q[kAhead];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (ES == 2) { x[2 * j] = __uint_as_float(w[j] << 16); x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
-            else x[j] = __uint_as_float(w[j]);
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < VEC; ++j) x[j] = (base + j < a.V) ? load_logit<ES>(row_base, base + j) : NINF;
+        for (int u = 0; u < kAhead; ++u) {
+          const unsigned i = i0 + 32u * u;
+          base[u] = i < n_g ? (int)my_groups[i] : -1;
+          q[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (base[u] >= 0 && base[u] + VEC <= v_main)       // a whole 16-byte piece of an aligned row
+            q[u] = __ldg(reinterpret_cast<const uint4*>(row_base + (size_t)base[u] * ES));
         }
-        unsigned n_c = 0u;
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) n_c += (x[j] >= cut_x) ? 1u : 0u;
-        unsigned at = atomicAdd(&seg_n[warp], n_c);
+        for (int u = 0; u < kAhead; ++u) {
+          if (base[u] < 0) continue;
+          float x[VEC];
+          if (base[u] + VEC <= v_main) {
+            const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-          if (!(x[j] >= cut_x)) continue;
-          if (at < (unsigned)kFiltSeg) my_seg[at] = make_uint2((unsigned)(base + j), bits_of(x[j]));
-          else sh_overflow = 1;
-          ++at;
+            for (int j = 0; j < 4; ++j) {
+              if (ES == 2) { x[2 * j] = __uint_as_float(w[j] << 16); x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
+              else x[j] = __uint_as_float(w[j]);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) x[j] = (base[u] + j < a.V) ? load_logit<ES>(row_base, base[u] + j) : NINF;
+          }
+          unsigned n_c = 0u;
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) n_c += (x[j] >= cut_x) ? 1u : 0u;
+          unsigned at = atomicAdd(&seg_n[warp], n_c);
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) {
+            if (!(x[j] >= cut_x)) continue;
+            if (at < (unsigned)kFiltSeg) my_seg[at] = make_uint2((unsigned)(base[u] + j), bits_of(x[j]));
+            else sh_overflow = 1;
+            ++at;
+          }
         }
       }
     }
