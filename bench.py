@@ -31,7 +31,10 @@ B_ROWS = 512
 VOCAB = 152064
 N_BUFFERS = 4                 # 4 x 155.7 MB of logits rotate, so no step finds its rows in the 126 MB L2
 ADV_B = 1024
-TRAFFIC_STEP_BYTES = 160.6e6  # dram bytes read + written per launch, ncu capture of this kernel at this workload (profiles/)
+# dram bytes read + written per launch of the step kernel at (B_ROWS, VOCAB, bf16, hierarchical sampler): a constant
+# copied from the ncu capture summarised under profiles/, not measured by this run
+TRAFFIC_STEP_BYTES = 160.6e6
+TARGET_REGION_MS = 150.0      # short timed regions are repeated until about this much device time has been timed
 
 PARAMS = dict(temperature=1.0, mu_g=6.0, sigma2_g=9.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0, eps=0.2,
               warmup_complete=1, t_max=1 << 30, eos_token=-1)
@@ -114,14 +117,14 @@ def cpu_threads() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_step_rate(rows_f32, values, seconds_target: float, sampler: int):
+def oracle_step_rate(rows_f32, values, seconds_target: float, sampler: int, cores: int | None = None):
     """Time the CPU oracle (as it stands) on a bounded sample of the benchmark's rows; returns rows/s.
 
-    The sample rows are advanced decode step after decode step (new draws each step) on all host
-    cores until about `seconds_target` seconds have passed.
+    The sample rows are advanced decode step after decode step (new draws each step) on `cores` threads (default:
+    all host cores) until about `seconds_target` seconds have passed.
     """
     import oracle
-    cores = cpu_threads()
+    cores = cores or cpu_threads()
     p = oracle.make_params(sampler=sampler, **PARAMS)
     n = rows_f32.shape[0]
     ro = oracle.Rollout(n, seed=1)
@@ -133,6 +136,17 @@ def oracle_step_rate(rows_f32, values, seconds_target: float, sampler: int):
         if dt >= seconds_target:
             break
     return done / dt, cores, done, dt
+
+
+def oracle_advantage_rate(r, v, L, s, n_traj: int, cores: int):
+    """Tokens/s of the oracle's advantage pass (backward recursion, float64) on the first `n_traj` trajectories."""
+    import numpy as np
+    import oracle
+    Ls = L[:n_traj]
+    n = int(Ls.astype(np.int64).sum())
+    t0 = time.perf_counter()
+    oracle.advantages_f32(r[:n], v[:n], Ls, s[:n_traj], 1.0, 0.95, -1.0, n_threads=cores)
+    return n / (time.perf_counter() - t0), n
 
 
 def run_reference(args):
@@ -181,6 +195,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the single-step timings at other shapes")
     ap.add_argument("--eager", action="store_true", help="launch every step separately instead of replaying a CUDA graph")
+    ap.add_argument("--repeats", type=int, default=None,
+                    help="times the K-step region is timed (default: enough repeats for ~150 ms; the median is reported)")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = args.steps or 4
@@ -231,7 +247,7 @@ def main():
         for i in range(n_steps):
             espo.espo_step(bufs[i % N_BUFFERS], values, state, params, tokens, stop)
 
-    # The decode loop is launch-latency sensitive (one 35 us kernel per step), so the timed rollout replays a CUDA
+    # The decode loop is launch-latency sensitive (one ~30 us kernel per step), so the timed rollout replays a CUDA
     # graph of GRAPH_STEPS consecutive steps (the remainder, and everything with --eager, is launched one by one).
     graph, graph_steps = None, 0
     if not args.eager and K >= 2 * N_BUFFERS:
@@ -259,32 +275,49 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    def region(ev):
+        """One timed region: K decode steps, then the advantage pass over the tokens they generated."""
+        ev[0].record()
+        timed_rollout(K)
+        ev[1].record()
+        espo.espo_advantages(adv_r, adv_v, adv_len, adv_stopped, 1.0, 0.95, -1.0, adv_out)
+        ev[2].record()
+
+    # Warm-up: W eager steps, then one untimed pass of exactly what is timed (so the graph that is timed has been
+    # replayed before), which also gives the region's duration.
     rollout(W)
-    espo.espo_advantages(adv_r, adv_v, adv_len, adv_stopped, 1.0, 0.95, -1.0, adv_out)
+    ev_w = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    region(ev_w)
+    torch.cuda.synchronize()
+    est_ms = max(ev_w[0].elapsed_time(ev_w[2]), 1e-3)
+    # A region of K steps that lasts less than TARGET_REGION_MS is repeated back to back (R times, every repeat
+    # timed by its own events) and the median repeat is reported: one 0.6 ms region is shorter than a clock sample
+    # and at the mercy of whatever the GPU did just before.
+    R = int(min(1000, max(1, round(TARGET_REGION_MS / est_ms)))) if args.repeats is None else max(1, args.repeats)
+    if dist is not None:
+        R = int(shard.max_over_ranks([R], dist, device=dev)[0])
     espo.espo_reset_state(state, 0)
     sampler_proc = ClockSampler(local_rank) if rank == 0 else None
     if sampler_proc:
         sampler_proc.start()
         time.sleep(0.3)
     barrier()
-    ev0, ev1, ev2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(R)]
     t_wall0 = time.time()
-    ev0.record()
-    timed_rollout(K)
-    ev1.record()
-    espo.espo_advantages(adv_r, adv_v, adv_len, adv_stopped, 1.0, 0.95, -1.0, adv_out)
-    ev2.record()
+    for ev in evs:
+        region(ev)
     barrier()
     t_wall1 = time.time()
-    ms_total = ev0.elapsed_time(ev2)
-    ms_steps = ev0.elapsed_time(ev1)
+    tot = sorted(ev[0].elapsed_time(ev[2]) for ev in evs)
+    stp = sorted(ev[0].elapsed_time(ev[1]) for ev in evs)
+    ms_total, ms_steps = statistics.median(tot), statistics.median(stp)
     ms_total, ms_steps = shard.max_over_ranks([ms_total, ms_steps], dist, device=dev)
     if sampler_proc:
         time.sleep(0.1)
         sampler_proc.stop()
     dev_status = espo.espo_state_status(state) | espo.espo_advantages_status()
     n_stopped = int((view["status"] != espo.ESPO_ROW_ACTIVE).sum().item())
-    assert int(view["t"].min().item()) == K or n_stopped > 0, "the timed rollout did not advance every trajectory"
+    assert int(view["t"].min().item()) == K * R or n_stopped > 0, "the timed rollout did not advance every trajectory"
 
     rows_per_s = world * B * K / (ms_total * 1e-3)
     bytes_per_launch = B * V * 2
@@ -292,6 +325,7 @@ def main():
     peak, peak_kind = measured_peaks()
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
 
+    traffic_known = (B == B_ROWS and args.sampler == "hier")
     out = {
         "metric": "fused ESPO step logit rows/s at V=152064 bf16", "value": rows_per_s, "unit": "rows/s",
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True,
@@ -300,15 +334,24 @@ def main():
             "workload": f"rollout-batch scale: B={B} trajectories per GPU, V={V}, bf16 logits ~N(0,3) + 5 Zipf peaks, "
                         f"temperature 1.0, {args.sampler} Philox Gumbel-max sampler, full active set; timed region = "
                         f"{K} decode steps + 1 advantage pass over the {adv_tokens} tokens generated",
-            "launch": ("eager launches" if graph is None else f"CUDA graph of {graph_steps} steps replayed"),
+            "logits_dtype": "bf16", "arithmetic": "f32 (f64 for the advantage scan's composition)",
+            "launch": ("eager launches" if graph is None else f"CUDA graph of {graph_steps} steps, replayed once before timing"),
             "l2": f"{N_BUFFERS} logit buffers of {bytes_per_launch / 1e6:.1f} MB rotate (each larger than the 126 MB L2)",
             "parallelism": f"rows sharded over {world} GPU(s), no collective",
             "stopped_rows": n_stopped, "device_status": dev_status,
         },
+        "timing": {"repeats": R, "region_ms_median": ms_total, "region_ms_min": tot[0], "region_ms_max": tot[-1],
+                   "steps_ms_median": ms_steps, "steps_ms_min": stp[0], "steps_ms_max": stp[-1],
+                   "note": "the K-step region (+ advantage pass) is timed `repeats` times back to back, each by its own "
+                           "CUDA events; value, ms_per_step and roofline use the median repeat (max over ranks)"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC_STEP_BYTES, "kernel": "espo_step_kernel<bf16,hier,bulk>",
+                     "traffic": TRAFFIC_STEP_BYTES if traffic_known else None,
+                     "traffic_source": ("constant from the ncu capture summarised under profiles/ (same kernel, same workload), "
+                                        "not measured by this run") if traffic_known else "no capture at this shape",
+                     "kernel": f"espo_step_kernel<bf16,{args.sampler},bulk>",
                      "peak_kind": f"of {peak_kind} copy bandwidth", "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "launch_us": kernel_ms * 1e3, "bytes_per_launch": bytes_per_launch},
+                     "launch_us": kernel_ms * 1e3, "launch_us_min": stp[0] / K * 1e3, "launch_us_max": stp[-1] / K * 1e3,
+                     "bytes_per_launch": bytes_per_launch},
         "gpu_launches": K + 2,
     }
 
@@ -399,36 +442,62 @@ def main():
             out["library_ops_same_bytes"] = lib
             del half, adv_src, adv_dst
 
-        # ---- single-step bandwidth at other shapes (the large-batch sweep; rotating buffers larger than 2x L2) ----
+        # Times launch(i) (i picks the input variant, so that consecutive launches read different buffers) as a CUDA
+        # graph of >= 40 launches: replayed once untimed, then for about 30 ms; returns microseconds per launch.
+        def graph_time_us(launch, n_variants, total_ms=30.0):
+            n = n_variants * max(1, -(-40 // n_variants))
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                for i in range(max(3, n_variants)):
+                    launch(i)
+                with torch.cuda.graph(g, stream=side):
+                    for i in range(n):
+                        launch(i)
+            torch.cuda.current_stream().wait_stream(side)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g.replay(); e1.record()
+            torch.cuda.synchronize()
+            reps = int(min(200, max(1, round(total_ms / max(e0.elapsed_time(e1), 1e-3)))))
+            e0.record()
+            for _ in range(reps):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / (reps * n)
+            del g
+            return us
+
+        # ---- single-step bandwidth at other shapes: the large-batch sweep, every (B, V, dtype) with the hierarchical
+        #      sampler and the V=152064 column with the flat one too; rotating buffers of > 2 x L2 in total ----
         if not args.no_sweep:
             sweep = []
-            for (sB, sV, sdt) in ((256, VOCAB, torch.bfloat16), (1024, VOCAB, torch.bfloat16), (2048, VOCAB, torch.bfloat16),
-                                  (512, VOCAB, torch.float32), (512, 128256, torch.bfloat16), (2048, 32000, torch.bfloat16)):
-                es = 2 if sdt == torch.bfloat16 else 4
-                per = sB * sV * es
-                nb = max(2, int(280e6 // per) + 1)
-                sbufs = [synth.logits_batch(sB, sV, dtype=sdt, sd=3.0, seed=500 + i, device=dev) for i in range(nb)]
-                sst = espo.espo_init_state(sB, sV, seed=99)
-                sval = torch.full((sB,), 0.5, dtype=torch.bfloat16, device=dev)
-                stok = torch.empty(sB, dtype=torch.int32, device=dev)
-                sstop = torch.empty(sB, dtype=torch.uint8, device=dev)
-                for i in range(20):
-                    espo.espo_step(sbufs[i % nb], sval, sst, params, stok, sstop)
-                torch.cuda.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                reps = 200
-                e0.record()
-                for i in range(reps):
-                    espo.espo_step(sbufs[i % nb], sval, sst, params, stok, sstop)
-                e1.record()
-                torch.cuda.synchronize()
-                us = e0.elapsed_time(e1) * 1e3 / reps
-                gbs = per / us / 1e3
-                sweep.append({"B": sB, "V": sV, "logits": "bf16" if es == 2 else "f32", "us": us, "GB/s": gbs,
-                              "frac_of_measured_peak": gbs / peak, "rows/s": sB / (us * 1e-6)})
-                espo.espo_free_state(sst)
-                del sbufs
-            out["bandwidth_sweep"] = sweep
+            flat_params = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, **PARAMS)
+            hier_params = espo.make_params(sampler=espo.ESPO_SAMPLER_HIER, **PARAMS)
+            for sV in (32000, 128256, VOCAB):
+                for sdt in (torch.bfloat16, torch.float32):
+                    for sB in (128, 256, 512, 1024, 2048):
+                        es = 2 if sdt == torch.bfloat16 else 4
+                        per = sB * sV * es
+                        nb = max(2, int(280e6 // per) + 1)
+                        sbufs = [synth.logits_batch(sB, sV, dtype=sdt, sd=3.0, seed=500 + i, device=dev) for i in range(nb)]
+                        sst = espo.espo_init_state(sB, sV, seed=99)
+                        sval = torch.full((sB,), 0.5, dtype=torch.bfloat16, device=dev)
+                        stok = torch.empty(sB, dtype=torch.int32, device=dev)
+                        sstop = torch.empty(sB, dtype=torch.uint8, device=dev)
+                        row = {"B": sB, "V": sV, "logits": "bf16" if es == 2 else "f32", "MB": per / 1e6}
+                        for name, pp in (("hier", hier_params),) + ((("flat", flat_params),) if sV == VOCAB else ()):
+                            us = graph_time_us(lambda i: espo.espo_step(sbufs[i % nb], sval, sst, pp, stok, sstop), nb)
+                            gbs = per / us / 1e3
+                            row[name] = {"us": us, "GB/s": gbs, "frac_of_measured_peak": gbs / peak,
+                                         "frac_of_nominal_8TBs": gbs / 8000.0, "rows/s": sB / (us * 1e-6)}
+                        sweep.append(row)
+                        espo.espo_free_state(sst)
+                        del sbufs
+            out["bandwidth_sweep"] = {"shapes": sweep,
+                                      "note": "one espo_step per launch, CUDA graph of >= 40 launches over rotating buffers "
+                                              "(> 280 MB in total), full active set; GB/s = B*V*sizeof(logit) / time"}
 
             # ---- shrinking active set: as rows stop, the caller passes the n_active surviving rows (compacted
             #      logits plus the slot list from espo_compact_active); per-step time vs n_active ----
@@ -438,57 +507,38 @@ def main():
             n_act_dev = torch.zeros(1, dtype=torch.int32, device=dev)
             for n_act in (B, (3 * B) // 4, B // 2, B // 4, B // 8):
                 ids = all_ids[:n_act].contiguous()
-                for i in range(10):
-                    espo.espo_step(bufs[i % N_BUFFERS][:n_act], values[:n_act], sst, params, tokens, stop, row_ids=ids, n_rows=n_act)
-                torch.cuda.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                reps = 200
-                e0.record()
-                for i in range(reps):
-                    espo.espo_step(bufs[i % N_BUFFERS][:n_act], values[:n_act], sst, params, tokens, stop, row_ids=ids, n_rows=n_act)
-                e1.record()
-                torch.cuda.synchronize()
-                us = e0.elapsed_time(e1) * 1e3 / reps
+                us = graph_time_us(lambda i: espo.espo_step(bufs[i % N_BUFFERS][:n_act], values[:n_act], sst, params, tokens, stop,
+                                                            row_ids=ids, n_rows=n_act), N_BUFFERS)
                 act.append({"n_active": n_act, "us": us, "GB/s": n_act * V * 2 / us / 1e3, "rows/s": n_act / (us * 1e-6)})
             ids_out = torch.empty(B, dtype=torch.int32, device=dev)
-            e0.record()
-            for _ in range(100):
-                espo.espo_compact_active(sst, ids_out, n_act_dev)
-            e1.record()
-            torch.cuda.synchronize()
-            out["active_set"] = {"steps": act, "compact_us": e0.elapsed_time(e1) * 1e3 / 100,
-                                 "note": f"capacity {B} slots, bf16, V={V}; eager launches; compaction is a separate one-CTA kernel"}
+            out["active_set"] = {"steps": act,
+                                 "compact_us": graph_time_us(lambda i: espo.espo_compact_active(sst, ids_out, n_act_dev), 1),
+                                 "note": f"capacity {B} slots, bf16, V={V}; CUDA graphs; compaction is a separate one-CTA kernel"}
             espo.espo_free_state(sst)
 
-        # ---- the other routes through the step: flat sampler, top-p filter, vocabulary shards (eager launches) ----
+        # ---- the other routes through the step: flat sampler, top-p filter, vocabulary shards ----
         if not args.no_sweep:
-            def step_us(p, reps, fn=None):
+            def step_us(p, fn=None, n_var=N_BUFFERS):
                 sst = espo.espo_init_state(B, V, seed=5)
-                call = fn or (lambda i: espo.espo_step(bufs[i % N_BUFFERS], values, sst, p, tokens, stop))
-                for i in range(3):
-                    call(i) if fn is None else fn(i, sst)
-                torch.cuda.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                for i in range(reps):
-                    call(i) if fn is None else fn(i, sst)
-                e1.record()
-                torch.cuda.synchronize()
+                call = (lambda i: espo.espo_step(bufs[i % N_BUFFERS], values, sst, p, tokens, stop)) if fn is None else (lambda i: fn(i, sst))
+                us = graph_time_us(call, n_var)
                 espo.espo_free_state(sst)
-                return e0.elapsed_time(e1) * 1e3 / reps
+                return us
             flat = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, **PARAMS)
             top_p = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, top_p=0.7, **PARAMS)
+            top_p_wide = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, top_p=0.9999, **PARAMS)
             cuts = shard.vocab_shards(V, 8)
             lo, n_ids = cuts[3]
             shard_bufs = [synth.logits_batch(B, n_ids, dtype=torch.bfloat16, sd=3.0, seed=700 + i, device=dev) for i in range(16)]
             parts = torch.zeros(8, B, 8, dtype=torch.float32, device=dev)
             out["other_routes"] = {
-                "flat_sampler_us": step_us(flat, 20),
-                "top_p_0.7_us": step_us(top_p, 40),
-                "vocab_shard_partial_us": step_us(flat, 100, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, flat, parts[3])),
-                "vocab_shard_merge_us": step_us(flat, 100, lambda i, sst: espo.espo_step_merge(parts, values, sst, flat, tokens, stop)),
-                "note": f"same batch (B={B}, V={V}, bf16); partial: one of 8 shards ({n_ids} ids) as its own buffer; merge: 8 x {B} "
-                        f"partials (host-bound when launched eagerly from Python)",
+                "flat_sampler_us": step_us(flat),
+                "top_p_0.7_us": step_us(top_p),
+                "top_p_0.9999_us": step_us(top_p_wide),
+                "vocab_shard_partial_us": step_us(flat, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, flat, parts[3]), 16),
+                "vocab_shard_merge_us": step_us(flat, lambda i, sst: espo.espo_step_merge(parts, values, sst, flat, tokens, stop), 1),
+                "note": f"same batch (B={B}, V={V}, bf16), CUDA graphs; partial: one of 8 shards ({n_ids} ids) as its own buffer; "
+                        f"merge: 8 x {B} partials",
             }
             del shard_bufs
 
@@ -529,10 +579,22 @@ def main():
         # ---- the CPU oracle on this machine's host cores, on a bounded sample of the same rows ----
         if not args.no_cpu_baseline:
             sample_src = bufs[0][:256].float().cpu().numpy()
-            rate, cores, n_rows, secs = oracle_step_rate(sample_src, np.full(256, 0.5), 12.0, sampler)
+            rate, cores, n_rows, secs = oracle_step_rate(sample_src, np.full(256, 0.5), 10.0, sampler)
             out["cpu_baseline"] = {"value": rate, "unit": "rows/s", "cores": cores, "kind": "oracle",
                                    "sample": f"{n_rows} row-steps: rows 0..255 of buffer 0 advanced step after step "
                                              f"for {secs:.1f} s on {cores} threads"}
+            rate1, _, n1, secs1 = oracle_step_rate(sample_src[:16], np.full(16, 0.5), 3.0, sampler, cores=1)
+            out["cpu_baseline"]["one_core"] = {"value": rate1, "unit": "rows/s", "cores": 1,
+                                               "sample": f"{n1} row-steps: rows 0..15 of buffer 0 for {secs1:.1f} s on 1 thread"}
+            # the oracle's advantage pass on a bounded slice of the advantage workload (tokens/s)
+            ar, av, aL, a_s = (t.cpu().numpy() for t in synth.ragged_trajectories(ADV_B, seed=0, device=dev))
+            a_all, n_all = oracle_advantage_rate(ar, av, aL, a_s, 256, cores)
+            a_one, n_one = oracle_advantage_rate(ar, av, aL, a_s, 64, 1)
+            out["cpu_baseline"]["advantages"] = {
+                "value": a_all, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                "sample": f"first 256 of the {ADV_B} trajectories of the advantage workload ({n_all} tokens), backward recursion "
+                          f"in float64, gamma=1, lambda=0.95",
+                "one_core": {"value": a_one, "unit": "tokens/s", "cores": 1, "sample": f"first 64 trajectories ({n_one} tokens)"}}
         print(json.dumps(out))
     espo.espo_free_state(state)
     if dist is not None:

@@ -1454,7 +1454,7 @@ struct espo_state {
   double* sum_h;
   float4* records;
   unsigned *ticket, *dev_status;
-  double* batch_out;   // [8] result of espo_end_batch
+  double* batch_out;   // [9] result of espo_end_batch
 };
 
 namespace espo {
@@ -1489,7 +1489,7 @@ __global__ void espo_compact_kernel(const uint8_t* __restrict__ status, int capa
 
 // Batch boundary (Eq. 7-8, 12): reduces the per-slot sums over the slots that took part (t > 0) and applies the
 // EMA and the proportional controller.  One CTA; out = {mu_g, sigma2_g, beta, mean, var, rho_stop, tokens,
-// trajectories} -- stopped trajectories = rho_stop * trajectories.
+// trajectories, stopped trajectories}.
 struct EndBatchArgs {
   const double *sum_g, *sum_g2;
   const int32_t* t;
@@ -1540,7 +1540,7 @@ __global__ void __launch_bounds__(1024) espo_end_batch_kernel(const EndBatchArgs
         beta = fmin(fmax(beta + e.eta_beta * (rho - e.tau), e.beta_min), e.beta_max);
       }
       e.out[0] = mu; e.out[1] = s2; e.out[2] = beta; e.out[3] = mean; e.out[4] = var; e.out[5] = rho;
-      e.out[6] = acc[2]; e.out[7] = acc[3];
+      e.out[6] = acc[2]; e.out[7] = acc[3]; e.out[8] = acc[4];
     }
   }
 }
@@ -1592,7 +1592,7 @@ int espo_init_state(espo_state** out, int32_t capacity, int32_t V, uint64_t seed
   const size_t o_t = carve(4 * cap), o_ts = carve(4 * cap), o_st = carve(cap);
   const size_t o_sg = carve(8 * cap), o_sg2 = carve(8 * cap), o_h = carve(4 * cap), o_sh = carve(8 * cap);
   const size_t o_rec = carve(sizeof(float4) * cap * (size_t)st->nblk);
-  const size_t o_tk = carve(4 * cap), o_ds = carve(4), o_bo = carve(8 * 8);
+  const size_t o_tk = carve(4 * cap), o_ds = carve(4), o_bo = carve(8 * 9);
   st->arena_bytes = off;
   e = cudaMalloc(&st->arena, st->arena_bytes);
   if (e != cudaSuccess) { delete st; return record_cuda_error(e); }
@@ -1611,6 +1611,11 @@ int espo_init_state(espo_state** out, int32_t capacity, int32_t V, uint64_t seed
                                  st->max_smem);
         if (e != cudaSuccess) { cudaFree(st->arena); delete st; return record_cuda_error(e); }
       }
+  // (the attribute belongs to the device that is current, so it is set for every state rather than once per process)
+  e = cudaFuncSetAttribute((const void*)espo_filtered_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFiltSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute((const void*)espo_filtered_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFiltSmemBytes);
+  if (e != cudaSuccess) { cudaFree(st->arena); delete st; return record_cuda_error(e); }
   int rc = reset_arrays(st, (cudaStream_t)stream);
   if (rc != ESPO_OK) { cudaFree(st->arena); delete st; return rc; }
   *out = st;
@@ -1698,6 +1703,11 @@ static int step_launch(const void* logits, int32_t logits_dtype, int64_t row_str
     if (rc != ESPO_OK) return rc;
   }
   if (n_rows == 0) return ESPO_OK;
+  {
+    int dev = -1;
+    ESPO_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != st->device) return ESPO_ERR_BAD_PARAM;      // the state lives on the device that was current at its creation
+  }
   if (!logits) return ESPO_ERR_NULL;
   if (!partial_out && (!values || !tokens_out || !stop_out)) return ESPO_ERR_NULL;
   if (row_stride < v_eff) return ESPO_ERR_BAD_SHAPE;
@@ -1768,12 +1778,7 @@ static int step_launch(const void* logits, int32_t logits_dtype, int64_t row_str
     // filtered sampling: its own kernel, one CTA per row
     if (p->sampler != ESPO_SAMPLER_FLAT || partial_out) return ESPO_ERR_BAD_PARAM;
     if (v_eff > (1 << 21)) return ESPO_ERR_CAPACITY;       // the histogram limbs are sized for rows up to 2^21 logits
-    static bool attr_set[2] = {false, false};
     auto fk = (es == 2) ? espo_filtered_kernel<2> : espo_filtered_kernel<4>;
-    if (!attr_set[es == 2]) {
-      ESPO_CUDA_TRY(cudaFuncSetAttribute((const void*)fk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFiltSmemBytes));
-      attr_set[es == 2] = true;
-    }
     const int fgrid = n_rows < st->sm_count ? n_rows : st->sm_count;
     fk<<<(unsigned)fgrid, kFiltThreads, kFiltSmemBytes, (cudaStream_t)stream>>>(a);
     ESPO_CUDA_TRY(cudaGetLastError());
@@ -1916,7 +1921,7 @@ int espo_end_batch(espo_state* st, float alpha_ema, float eta_beta, float tau, f
   cudaStream_t s = (cudaStream_t)stream;
   espo::espo_end_batch_kernel<<<1, 1024, 0, s>>>(e);
   ESPO_CUDA_TRY(cudaGetLastError());
-  double host[8];
+  double host[9];
   ESPO_CUDA_TRY(cudaMemcpyAsync(host, st->batch_out, sizeof(host), cudaMemcpyDeviceToHost, s));
   ESPO_CUDA_TRY(cudaStreamSynchronize(s));
   params_inout->mu_g = (float)host[0];
@@ -1924,7 +1929,7 @@ int espo_end_batch(espo_state* st, float alpha_ema, float eta_beta, float tau, f
   params_inout->beta = (float)host[2];
   if (stats_out) {
     stats_out[0] = host[3]; stats_out[1] = host[4]; stats_out[2] = host[5];
-    stats_out[3] = host[6]; stats_out[4] = host[7]; stats_out[5] = host[5] * host[7];
+    stats_out[3] = host[6]; stats_out[4] = host[7]; stats_out[5] = host[8];
   }
   return ESPO_OK;
 }

@@ -1,4 +1,4 @@
-"""espo_advantages_noalloc against espo_advantages, through the C ABI (needs a B200).
+"""espo_advantages_noalloc against espo_advantages and against the CPU oracle, through the C ABI (needs a B200).
 
 The entry point exists for processes that cannot allocate device memory once they are running --
 a rollout worker whose serving engine took all free memory for its own pools, or a loop that
@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2605_29860_b200 as espo
 from paper_2605_29860_b200 import synth
 
@@ -28,6 +29,13 @@ def _both(r, v, L, s, gamma, lam, r_fail, status):
     ref, got = ref.cpu().numpy().astype(np.float64), got.cpu().numpy().astype(np.float64)
     bad = np.nonzero(~(np.abs(got - ref) <= ATOL + RTOL * np.abs(ref)))[0]
     assert bad.size == 0, f"{bad.size} of {ref.size} differ, first at {bad[:5]}: {got[bad[:5]]} vs {ref[bad[:5]]}"
+    # and against the CPU oracle (Eq. 4-5, 13 in float64), the checker of every other advantage test;
+    # the C ABI takes gamma, lambda and r_fail as float32, so the oracle gets the same numbers
+    f32 = lambda x: float(np.float32(x))
+    want = oracle.advantages(r.cpu().numpy(), v.cpu().numpy(), L.cpu().numpy(), s.cpu().numpy(), f32(gamma), f32(lam),
+                             f32(r_fail))
+    bad = np.nonzero(~(np.abs(got - want) <= ATOL + RTOL * np.abs(want)))[0]
+    assert bad.size == 0, f"{bad.size} of {want.size} differ from the oracle, first at {bad[:5]}: {got[bad[:5]]} vs {want[bad[:5]]}"
 
 
 def test_two_calls_in_a_row_match_the_allocating_entry_point():
