@@ -10,7 +10,7 @@ _CSRC = os.path.join(_PKG, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_PKG, "libespo.so")
 SOURCES = ["espo_api.cu", "espo_step.cu", "espo_adv.cu"]
-HEADERS = ["espo_device.cuh", "espo_host.h"]
+HEADERS = ["espo_device.cuh", "espo_host.h", "espo_step_common.cuh", "espo_step_hier.cuh"]
 
 
 def _nvcc() -> str:

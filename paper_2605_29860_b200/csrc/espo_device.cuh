@@ -111,6 +111,11 @@ __device__ __forceinline__ uint4 ld_volatile_u4(const uint4* p) {
 __device__ __forceinline__ void st_volatile_u4(uint4* p, uint4 v) {
   asm volatile("st.volatile.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+__device__ __forceinline__ int2 ld_volatile_i2(const void* p) {
+  int2 v;
+  asm volatile("ld.volatile.v2.s32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ float4 ld_volatile_f4(const void* p) {
   float4 v;
   asm volatile("ld.volatile.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
