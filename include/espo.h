@@ -182,6 +182,14 @@ int espo_state_view(espo_state* st, const float** z, const float** g, const floa
  * Errors: NULL, BAD_PARAM. */
 int espo_set_launch_config(espo_state* st, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm);
 
+/* Programmatic dependent launch for the step kernel of ESPO_SAMPLER_HIER (the paper has no counterpart; it is how a
+ * decode loop hides launch latency on this hardware).  With enable != 0, espo_step launches its kernel so that the
+ * GPU may set it up -- place its thread blocks, run the part that touches no global memory -- while the kernel
+ * that precedes it in the stream is still finishing; the step kernel waits for that kernel's completion before it
+ * reads or writes any global memory, so what it computes does not change.  The step kernel in turn lets a
+ * kernel launched after it in the same way start early.  Off by default.  Errors: NULL. */
+int espo_set_dependent_launch(espo_state* st, int32_t enable);
+
 /* Stable compaction of the active set: writes the slots whose status is ESPO_ROW_ACTIVE, in
  * increasing order, to row_ids_out (device int32 [capacity]) and their number to
  * n_active_out (device int32 [1]).  Enqueued on `stream`. */

@@ -72,6 +72,7 @@ def lib():
         L.espo_free_state.argtypes = [vp]
         L.espo_free_state.restype = None
         L.espo_set_launch_config.argtypes = [vp, i32, i32, i32]
+        L.espo_set_dependent_launch.argtypes = [vp, i32]
         L.espo_step.argtypes = [vp, i32, i64, vp, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp, vp]
         L.espo_step_partial.argtypes = [vp, i32, i64, i32, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp]
         L.espo_step_merge.argtypes = [vp, i32, i64, vp, i32, vp, i32, vp, C.POINTER(espo_params), vp, vp, vp]
@@ -166,6 +167,11 @@ def espo_free_state(state: EspoState) -> None:
 
 def espo_set_launch_config(state: EspoState, consumer_warps: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
     _check(lib().espo_set_launch_config(state.handle, consumer_warps, stages, ctas_per_sm), "espo_set_launch_config")
+
+
+def espo_set_dependent_launch(state: EspoState, enable: bool = True) -> None:
+    """Let the hierarchical step kernel be set up while the kernel before it in the stream winds down; see ``espo.h``."""
+    _check(lib().espo_set_dependent_launch(state.handle, int(bool(enable))), "espo_set_dependent_launch")
 
 
 def espo_step(logits: torch.Tensor, values: torch.Tensor, state: EspoState, params: espo_params,

@@ -1096,6 +1096,7 @@ struct espo_state {
   int device, capacity, V, nblk, sm_count, max_smem;
   uint64_t seed, batch_id;
   int cfg_warps, cfg_stages, cfg_ctas_per_sm;   // 0 = library default
+  int dependent_launch;                         // espo_set_dependent_launch
   void* arena;
   size_t arena_bytes;
   float *z, *g, *g_tilde, *logp;
@@ -1306,6 +1307,12 @@ int espo_set_launch_config(espo_state* st, int32_t consumer_warps, int32_t stage
   return ESPO_OK;
 }
 
+int espo_set_dependent_launch(espo_state* st, int32_t enable) {
+  if (!st) return ESPO_ERR_NULL;
+  st->dependent_launch = enable != 0;
+  return ESPO_OK;
+}
+
 // Checks the frozen parameters and digests them into the kernel's arguments (everything but shapes and pointers).
 static int fill_params(espo::StepArgs& a, const espo_state* st, const espo_params* p) {
   using namespace espo;
@@ -1360,8 +1367,11 @@ static int launch_hier(espo::StepArgs& a, const espo_state* st, int es, bool bul
   int stages = st->cfg_stages ? st->cfg_stages : 2;
   if (warps + fin > max_warps) warps = max_warps - fin;
   if (warps < 1) warps = 1;
+  if (a.total_blocks >= (1ll << 31)) return 1;
   long long grid = (long long)st->sm_count * ctas_per_sm;
   if (grid > a.total_blocks) grid = a.total_blocks;
+  a.blk_base = (int)(a.total_blocks / grid);
+  a.blk_rem = (int)(a.total_blocks % grid);
   const long long blocks_per_cta = (a.total_blocks + grid - 1) / grid;
   if (blocks_per_cta < warps) warps = (int)blocks_per_cta;
   const long long rows = blocks_per_cta / a.nblk + 2;      // rows a CTA's range can touch
@@ -1397,10 +1407,23 @@ static int launch_hier(espo::StepArgs& a, const espo_state* st, int es, bool bul
   a.fin_warps = fin;
   a.stages = stages;
   a.run_len = (a.nblk >= 64) ? 1 : (a.nblk >= 32 ? 4 : (a.nblk >= 8 ? 2 : 1));
+  for (int i = 0; i < 2; ++i) {
+    const int n_runs = (a.blk_base + i + a.run_len - 1) / a.run_len;
+    a.runs_q[i] = n_runs / warps;
+    a.runs_r[i] = n_runs % warps;
+  }
   auto k = (es == 2) ? (bulk ? espo_step_hier_kernel<2, true> : espo_step_hier_kernel<2, false>)
                      : (bulk ? espo_step_hier_kernel<4, true> : espo_step_hier_kernel<4, false>);
-  k<<<(unsigned)grid, (unsigned)(warps + fin) * 32u, total, stream>>>(a);
-  ESPO_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)(warps + fin) * 32u);
+  cfg.dynamicSmemBytes = total;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may be set up while the kernel before it winds down
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  if (st->dependent_launch) { cfg.attrs = attr; cfg.numAttrs = 1; }
+  ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, k, a));
   return ESPO_OK;
 }
 

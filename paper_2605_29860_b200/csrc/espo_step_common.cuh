@@ -43,6 +43,8 @@ struct StepArgs {
   unsigned* dev_status; // sticky ESPO_DEV_* bits
   // shared-memory layout of the hierarchical kernel: byte offsets of its tables, laid out by the host
   int h_bars, h_meta, h_ctrl, h_ready, h_pre, h_noise, h_lrec, h_fscratch;
+  int blk_base, blk_rem;      // blocks per CTA: the first blk_rem CTAs take blk_base + 1, the others blk_base
+  int runs_q[2], runs_r[2];   // runs of run_len blocks in a range of blk_base (+1) blocks, divided by the streaming warps
   // frozen parameters, pre-digested on the host
   float inv_temp;       // 1/temperature (1 when greedy)
   float k2;             // inv_temp * log2(e)

@@ -486,23 +486,31 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_hier_kernel(cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  // The next kernel in the stream may be set up now (if it was launched as a programmatic dependent); this one reads
+  // or writes no global memory before the wait below.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  // The CTA's range: the first `blk_rem` CTAs take blk_base + 1 blocks, the others blk_base (fewer than 2^31 blocks in
+  // all: 32-bit arithmetic, a launch starts with cold instruction and constant caches and every subroutine counts).
   CtaRange cr;
+  const int big = (int)blockIdx.x < a.blk_rem;
   {
-    const long long g0 = (long long)blockIdx.x * a.total_blocks / gridDim.x;
-    const long long g1 = (long long)(blockIdx.x + 1) * a.total_blocks / gridDim.x;
+    const unsigned g0 = blockIdx.x * (unsigned)a.blk_base + (unsigned)min((int)blockIdx.x, a.blk_rem);
     cr.nblk = a.nblk;
-    cr.r_first = g0 / a.nblk;
-    cr.b0 = (int)(g0 - cr.r_first * a.nblk);
-    cr.n = (int)(g1 - g0);
-    const long long r_last = (g1 - 1) / a.nblk;
-    cr.n_local = (int)(r_last - cr.r_first) + 1;
-    const long long last_start = r_last * a.nblk;       // the walk starts where the last row's part starts
-    cr.off = (last_start > g0) ? (int)(last_start - g0) : 0;
+    cr.n = a.blk_base + big;
+    const unsigned r_first = g0 / (unsigned)a.nblk;
+    cr.r_first = r_first;
+    cr.b0 = (int)(g0 - r_first * (unsigned)a.nblk);
+    const int last = cr.b0 + cr.n - 1;                  // the range's last block, counted from block 0 of its first row
+    const int k_last = last / a.nblk;
+    cr.n_local = k_last + 1;
+    cr.off = k_last > 0 ? k_last * a.nblk - cr.b0 : 0;  // the walk starts where the last row's part starts
   }
 
   if (warp >= W) {
     // ------------------------------------------------------------------ finalizer warps
     // the state of the first rows of the walk is asked for before anything else, ahead of the streaming warps' traffic
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the kernel before this one has completed
     RowPre first_pre;
     {
       const int idx = (warp - W) * 32 + lane;
@@ -518,7 +526,6 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_hier_kernel(cons
 
   // -------------------------------------------------------------------- streaming warps
   if (threadIdx.x == 0) { *abort_flag = 0; *next_row = 0; }
-  for (int i = threadIdx.x; i < cr.n; i += W * 32) tb.lrec[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   if (lane == 0) {
     for (int s = 0; s < S; ++s) mbar_init(&bars[warp * S + s], 1);
     mbar_init_fence();
@@ -529,14 +536,13 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_hier_kernel(cons
   int2* my_meta = metas + warp * S;            // (position in the range, block of its row) of the block each stage holds
   // The warps take turns of C consecutive positions of the CTA's walk: warp w owns the runs w, w + W, w + 2W, ...
   const int C = a.run_len;
-  int n_my = 0;
+  int n_my;
   {
-    const int n_runs = (cr.n + C - 1) / C;
-    if (n_runs > warp) {
-      const int mine = (n_runs - warp + W - 1) / W;            // runs owned by this warp
-      n_my = mine * C;
-      if ((n_runs - 1) % W == warp) n_my -= n_runs * C - cr.n;  // the walk's last run may be short
-    }
+    // runs of the walk = runs_q * W + runs_r (divided on the host, for either size of range)
+    const int q = a.runs_q[big], r = a.runs_r[big];
+    n_my = (q + (warp < r ? 1 : 0)) * C;
+    const int last_owner = r ? r - 1 : W - 1;                   // the walk's last run may be short
+    if (warp == last_owner && n_my > 0) n_my -= (q * W + r) * C - cr.n;
   }
   constexpr int kBlockBytes = kBlockIds * ES;
 
@@ -547,7 +553,7 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_hier_kernel(cons
   auto seek = [&](int q) {
     fq = q;
     const int li = cr.b0 + q;
-    const int lrow = li / cr.nblk;
+    const int lrow = (int)((unsigned)li / (unsigned)cr.nblk);
     f_blk = li - lrow * cr.nblk;
     f_ptr = a.logits + (size_t)(cr.r_first + lrow) * a.row_stride_bytes + (size_t)f_blk * kBlockBytes;
   };
@@ -576,12 +582,14 @@ __global__ void __launch_bounds__(kMaxStepThreads, 1) espo_step_hier_kernel(cons
     bulk_copy_g2s(my_ring + (size_t)s * a.stage_bytes, f_ptr, bytes, &my_bar[s]);
   };
   int fetched = 0;
+  asm volatile("griddepcontrol.wait;" ::: "memory");       // the kernel before this one has completed
   if (BULK) {
     for (; fetched < S && fetched < n_my; ++fetched) {
       if (lane == 0) issue(fetched);
       advance();
     }
   }
+  for (int i = threadIdx.x; i < cr.n; i += W * 32) tb.lrec[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   // (A) among the streaming warps: the record table is cleared before anybody writes a record; (B) tells the
   // finalizer warps so without waiting for them (they start with loads from global memory)
   asm volatile("bar.sync 1, %0;" ::"r"(W * 32) : "memory");
