@@ -195,6 +195,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the single-step timings at other shapes")
     ap.add_argument("--eager", action="store_true", help="launch every step separately instead of replaying a CUDA graph")
+    ap.add_argument("--no-dependent-launch", action="store_true",
+                    help="launch the step kernel plainly (default: as a programmatic dependent of the kernel before it)")
     ap.add_argument("--repeats", type=int, default=None,
                     help="times the K-step region is timed (default: enough repeats for ~150 ms; the median is reported)")
     args = ap.parse_args()
@@ -233,6 +235,11 @@ def main():
     tokens = torch.empty(B, dtype=torch.int32, device=dev)
     stop = torch.empty(B, dtype=torch.uint8, device=dev)
     state = espo.espo_init_state(B, V, seed=plan["state_seed"])
+    # The step kernel is launched as a programmatic dependent of whatever precedes it in the stream (in a decode loop:
+    # the LM head; here: the previous step): the GPU places its thread blocks and runs its set-up while that kernel
+    # winds down, and the kernel waits for that kernel's completion before it touches global memory.
+    use_pdl = not args.no_dependent_launch
+    espo.espo_set_dependent_launch(state, use_pdl)
     view = espo.espo_state_view(state)
     # rollout record for the closing advantage pass: K tokens per trajectory, reward 0 except the end
     adv_tokens = B * K
@@ -335,7 +342,9 @@ def main():
                         f"temperature 1.0, {args.sampler} Philox Gumbel-max sampler, full active set; timed region = "
                         f"{K} decode steps + 1 advantage pass over the {adv_tokens} tokens generated",
             "logits_dtype": "bf16", "arithmetic": "f32 (f64 for the advantage scan's composition)",
-            "launch": ("eager launches" if graph is None else f"CUDA graph of {graph_steps} steps, replayed once before timing"),
+            "launch": ("eager launches" if graph is None else f"CUDA graph of {graph_steps} steps, replayed once before timing")
+                      + ("; step kernel launched as a programmatic dependent (set-up overlaps the previous kernel's end, no "
+                         "global memory touched before that kernel has completed)" if use_pdl else "; plain launches"),
             "l2": f"{N_BUFFERS} logit buffers of {bytes_per_launch / 1e6:.1f} MB rotate (each larger than the 126 MB L2)",
             "parallelism": f"rows sharded over {world} GPU(s), no collective",
             "stopped_rows": n_stopped, "device_status": dev_status,
@@ -468,6 +477,16 @@ def main():
             us = e0.elapsed_time(e1) * 1e3 / (reps * n)
             del g
             return us
+
+        # ---- the bench's step under both launch modes, timed the same way (graph of 40 steps over the rotating buffers)
+        if not args.no_sweep:
+            modes = {}
+            for name, flag in (("plain_launch_us", False), ("dependent_launch_us", True)):
+                mst = espo.espo_init_state(B, V, seed=3)
+                espo.espo_set_dependent_launch(mst, flag)
+                modes[name] = graph_time_us(lambda i: espo.espo_step(bufs[i % N_BUFFERS], values, mst, params, tokens, stop), N_BUFFERS)
+                espo.espo_free_state(mst)
+            out["launch_modes"] = modes
 
         # ---- single-step bandwidth at other shapes: the large-batch sweep, every (B, V, dtype) with the hierarchical
         #      sampler and the V=152064 column with the flat one too; rotating buffers of > 2 x L2 in total ----

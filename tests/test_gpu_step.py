@@ -150,6 +150,32 @@ def test_results_do_not_depend_on_launch_shape_and_repeat_bit_exactly():
                 assert torch.equal(a, b)
 
 
+def test_dependent_launch_changes_nothing():
+    # espo_set_dependent_launch only lets the step kernel be set up early; several steps back to back (each the
+    # programmatic dependent of the one before) must leave exactly what plain launches leave
+    B, V, T = 300, 152064, 4
+    p = espo.make_params(temperature=1.0, mu_g=1.0, sigma2_g=2.0, beta=2.0)
+    xs = [synth.logits_batch(B, V, dtype=torch.bfloat16, seed=60 + t) for t in range(T)]
+    v = torch.rand(B, device="cuda")
+    outs = []
+    for flag in (False, True):
+        st = espo.espo_init_state(B, V, seed=11)
+        espo.espo_set_dependent_launch(st, flag)
+        toks = [torch.empty(B, dtype=torch.int32, device="cuda") for _ in range(T)]
+        stop = torch.empty(B, dtype=torch.uint8, device="cuda")
+        for t in range(T):
+            espo.espo_step(xs[t], v, st, p, toks[t], stop)
+        torch.cuda.synchronize()
+        view = espo.espo_state_view(st)
+        outs.append(([t.cpu() for t in toks], view["z"].cpu().clone(), view["logp"].cpu().clone(), view["t"].cpu().clone()))
+        assert espo.espo_state_status(st) == 0
+        espo.espo_free_state(st)
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert torch.equal(a, b)
+    assert all(torch.equal(a, b) for a, b in zip(outs[0][1:], outs[1][1:]))
+    assert int(outs[0][3].min()) >= 1
+
+
 # ---------------------------------------------------------------------------- special rows and rules
 
 
