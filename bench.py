@@ -546,7 +546,7 @@ def main():
             flat = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, **PARAMS)
             top_p = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, top_p=0.7, **PARAMS)
             top_p_wide = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT, top_p=0.9999, **PARAMS)
-            cuts = shard.vocab_shards(V, 8)
+            cuts = shard.vocab_shards(V, 8, multiple=1024)
             lo, n_ids = cuts[3]
             shard_bufs = [synth.logits_batch(B, n_ids, dtype=torch.bfloat16, sd=3.0, seed=700 + i, device=dev) for i in range(16)]
             parts = torch.zeros(8, B, 8, dtype=torch.float32, device=dev)
@@ -555,6 +555,7 @@ def main():
                 "top_p_0.7_us": step_us(top_p),
                 "top_p_0.9999_us": step_us(top_p_wide),
                 "vocab_shard_partial_us": step_us(flat, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, flat, parts[3]), 16),
+                "vocab_shard_partial_hier_us": step_us(params, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, params, parts[3]), 16),
                 "vocab_shard_merge_us": step_us(flat, lambda i, sst: espo.espo_step_merge(parts, values, sst, flat, tokens, stop), 1),
                 "note": f"same batch (B={B}, V={V}, bf16), CUDA graphs; partial: one of 8 shards ({n_ids} ids) as its own buffer; "
                         f"merge: 8 x {B} partials",

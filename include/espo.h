@@ -230,13 +230,19 @@ int espo_end_batch_merge(const double* stats, int32_t n_parts, float alpha_ema, 
  * (espo_step_partial), the partials of all shards are brought together (one all-gather of 32 bytes per row and
  * shard when the shards live on different GPUs; the library does not communicate) and espo_step_merge finishes the
  * step on the trajectory state: regret, normalisation, smoothing, stop rule, bookkeeping (Eq. 6, 9-11), exactly as
- * espo_step does.  Only the flat sampler is offered: its Gumbel draws belong to token ids, so the perturbed maximum
- * over the shards is the perturbed maximum over the row and the token does not depend on how the row is cut. */
+ * espo_step does.  With the flat sampler the Gumbel draws belong to token ids, so the perturbed maximum over the
+ * shards is the perturbed maximum over the row and the token does not depend on how the row is cut.  With the
+ * hierarchical sampler the block-level draws belong to blocks of 1024 ids of the whole vocabulary: shards that start
+ * on such a block give exactly the token of espo_step (each shard resolves the token inside its own best block and
+ * reports that block's perturbed score; the merge takes the best of them).  Greedy decoding (temperature 0) and the
+ * entropy are offered with the flat sampler only. */
 typedef struct espo_partial {
   float m;             /* largest logit of the shard's part of the row (-inf if it has no finite entry)           */
   float s;             /* sum over the part of exp((x - m) / temperature)                                          */
-  float best;          /* largest perturbed score x/T + G of the part (greedy: the largest logit)                  */
-  int32_t best_id;     /* global token id that attains it, lowest id on ties; -1: none                             */
+  float best;          /* largest perturbed score x/T + G of the part (greedy: the largest logit; hierarchical       */
+                       /* sampler: the best block's score m_b/T + ln s_b + G_b)                                     */
+  int32_t best_id;     /* global token id that attains it, lowest id on ties (hierarchical: the token drawn inside  */
+                       /* that block); -1: none                                                                     */
   float x_best;        /* that token's logit                                                                        */
   uint32_t flags;      /* bit 0: the part held NaN or +inf; bit 1: nothing computed (bad slot or ended trajectory) */
   uint32_t reserved[2];
@@ -246,9 +252,11 @@ typedef struct espo_partial {
  * partial_out; changes nothing else, so the shards of a step may run in any order or on different GPUs with
  * replicas of the state.
  *   logits_shard   device [n_rows, v_shard] with row_stride elements between rows, dtype as for espo_step
- *   vocab_offset   global id of the shard's first logit; a multiple of 4; vocab_offset + v_shard <= V
+ *   vocab_offset   global id of the shard's first logit; a multiple of 4 (ESPO_SAMPLER_HIER: of 1024);
+ *                  vocab_offset + v_shard <= V
  *   partial_out    device espo_partial [n_rows], 16-byte aligned
- *   params         sampler must be ESPO_SAMPLER_FLAT (else ESPO_ERR_BAD_PARAM); temperature 0 = greedy
+ *   params         either sampler; ESPO_SAMPLER_HIER needs temperature > 0 and want_entropy = 0 (else
+ *                  ESPO_ERR_BAD_PARAM); with ESPO_SAMPLER_FLAT temperature 0 = greedy
  * Calls that use the same state must not overlap on the device (they share its scratch).
  * Errors: NULL, BAD_SHAPE, BAD_DTYPE, BAD_PARAM, ALIGN, CAPACITY, CUDA. */
 int espo_step_partial(const void* logits_shard, int32_t logits_dtype, int64_t row_stride, int32_t v_shard,

@@ -1484,9 +1484,10 @@ static int step_launch(const void* logits, int32_t logits_dtype, int64_t row_str
     return ESPO_OK;
   }
   const bool bulk = ((uintptr_t)logits % 16 == 0) && (a.row_stride_bytes % 16 == 0) && (((size_t)v_eff * es) % 16 == 0);
-  if (p->sampler == ESPO_SAMPLER_HIER && !a.greedy && !partial_out) {
+  if (p->sampler == ESPO_SAMPLER_HIER && !a.greedy) {
     const int rc = launch_hier(a, st, es, bulk, (cudaStream_t)stream);
     if (rc != 1) return rc;
+    if (partial_out) return ESPO_ERR_CAPACITY;     // only that kernel serves shards of the hierarchical sampler
   }
   // Launch shape: ctas_per_sm CTAs of `warps` streaming warps (+1 finalizer warp), `stages` blocks in flight per warp.
   int ctas_per_sm = st->cfg_ctas_per_sm ? st->cfg_ctas_per_sm : 1;
@@ -1550,7 +1551,12 @@ int espo_step_partial(const void* logits_shard, int32_t logits_dtype, int64_t ro
                       espo_partial* partial_out, void* stream) {
   if (!st || !p) return ESPO_ERR_NULL;
   if (v_shard < 1 || vocab_offset < 0 || (vocab_offset & 3) || (long long)vocab_offset + v_shard > st->V) return ESPO_ERR_BAD_SHAPE;
-  if (p->sampler != ESPO_SAMPLER_FLAT) return ESPO_ERR_BAD_PARAM;   // the flat sampler's draws belong to ids, not to blocks of a row
+  if (p->sampler == ESPO_SAMPLER_HIER) {
+    // the hierarchical sampler's draws belong to blocks of 1024 ids of the whole vocabulary: a shard starts on one
+    if ((vocab_offset & 1023) || p->want_entropy || !(p->temperature > 0.f)) return ESPO_ERR_BAD_PARAM;
+  } else if (p->sampler != ESPO_SAMPLER_FLAT) {
+    return ESPO_ERR_BAD_PARAM;
+  }
   if (n_rows > 0 && !partial_out) return ESPO_ERR_NULL;
   return step_launch(logits_shard, logits_dtype, row_stride, nullptr, ESPO_F32, row_ids, n_rows, st, p, nullptr, nullptr,
                      v_shard, vocab_offset, partial_out, stream);
@@ -1570,7 +1576,7 @@ int espo_step_merge(const espo_partial* partials, int32_t n_shards, int64_t shar
     const int rc = fill_params(a, st, p);
     if (rc != ESPO_OK) return rc;
   }
-  if (p->sampler != ESPO_SAMPLER_FLAT) return ESPO_ERR_BAD_PARAM;
+  if (p->want_entropy) return ESPO_ERR_BAD_PARAM;      // the partials do not carry the entropy sums
   if (n_rows == 0) return ESPO_OK;
   if (!partials || !values || !tokens_out || !stop_out) return ESPO_ERR_NULL;
   const int ves = (values_dtype == ESPO_BF16) ? 2 : 4;

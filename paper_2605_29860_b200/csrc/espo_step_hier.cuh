@@ -98,6 +98,8 @@ __device__ __forceinline__ float stage_logit(const unsigned char* stage, int pos
 template <int ES>
 __device__ __forceinline__ void hier_descend_stage(const StepArgs& a, const unsigned char* stage, int nvalid, int blk,
                                                    uint32_t slot, uint32_t step, int lane, int& token, float& l_tok) {
+  // `blk` is the block's number in the whole vocabulary (a vocabulary shard starts at a multiple of 1024 ids): the
+  // draws belong to global sub-block and token numbers, and the token returned is a global id.
   const float NINF = __int_as_float(0xff800000);
   const DrawStream ds{a.key0, a.key1, step, slot, a.batch_bits};
   constexpr int kVecsPerSub = kSubIds * ES / 16;     // 16-byte vectors of a sub-block: 4 (bfloat16) or 8 (float32)
@@ -264,8 +266,29 @@ __device__ __forceinline__ void hier_resolve(const StepArgs& a, int row, int blk
                                              int lane, int& token, float& l_tok) {
   const int nvalid = min(kBlockIds, a.V - blk * kBlockIds);
   hier_fetch_block<ES>(a, a.logits + (size_t)row * a.row_stride_bytes, blk, nvalid, scratch, lane);
-  hier_descend_stage<ES>(a, scratch, nvalid, blk, (uint32_t)pre.slot, (uint32_t)pre.t_now, lane, token, l_tok);
+  hier_descend_stage<ES>(a, scratch, nvalid, blk + (a.vocab_offset >> 10), (uint32_t)pre.slot, (uint32_t)pre.t_now, lane, token, l_tok);
   __syncwarp();
+}
+
+// What a vocabulary shard leaves about a row instead of acting on it (espo_step_partial): flags bit 0: the shard's
+// part of the row held NaN or +inf; bit 1: nothing was computed because the slot is bad or the trajectory has ended.
+__device__ __forceinline__ void hier_report(const StepArgs& a, int row, int lane, float m, float s, float best, int token,
+                                            float l_tok, unsigned flags, bool no_ticket) {
+  if (lane == 0) {
+    espo_partial pr;
+    pr.m = m; pr.s = s; pr.best = best; pr.best_id = token; pr.x_best = l_tok; pr.flags = flags;
+    pr.reserved[0] = 0u; pr.reserved[1] = 0u;
+    a.partial_out[row] = pr;
+    if (!no_ticket) a.ticket[row] = 0;   // ready for the next launch
+  }
+}
+
+// A row whose slot is bad or whose trajectory has ended: untouched, token -1.
+__device__ __forceinline__ void hier_skip_row(const StepArgs& a, int row, int lane, const RowPre& pre, bool no_ticket) {
+  const float NINF = __int_as_float(0xff800000);
+  if (a.partial_out) hier_report(a, row, lane, NINF, 0.f, NINF, -1, NINF, 2u, no_ticket);
+  else if (pre.slot < 0) mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, no_ticket);
+  else mark_row(a, row, pre.slot, lane, -1, 0u, -1, no_ticket);
 }
 
 // The end of a row: merges the lanes' running values in a fixed order and commits the row (Eq. 6, 9, 10, 11).
@@ -298,12 +321,19 @@ __device__ __noinline__ void hier_commit(const StepArgs& a, int row, int lane, c
     if (a.want_entropy) run_u = warp_sum(run_u);
   }
   const float M = run_m, S = run_s;
+  if (a.partial_out) {
+    // a vocabulary shard: leave what the merge needs and do not touch the state (a shard may hold no finite logit)
+    if (poisoned || M == __int_as_float(0x7f800000) || M != M) hier_report(a, row, lane, NINF, 0.f, NINF, -1, NINF, 1u, no_ticket);
+    else if (best_b < 0) hier_report(a, row, lane, NINF, 0.f, NINF, -1, NINF, 0u, no_ticket);
+    else hier_report(a, row, lane, M, S, best, c_token, c_ltok, 0u, no_ticket);
+    return;
+  }
   if (poisoned || best_b < 0 || M == __int_as_float(0x7f800000) || M != M || !(M > NINF) || isinf(M)) {
     mark_row(a, row, slot, lane, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, no_ticket);
     return;
   }
   const DrawStream ds{a.key0, a.key1, (uint32_t)pre.t_now, (uint32_t)slot, a.batch_bits};
-  if (lane == 0) commit_row(a, row, pre, ds, M, S, logf(S), run_u, c_ltok, c_token + a.vocab_offset, no_ticket);
+  if (lane == 0) commit_row(a, row, pre, ds, M, S, logf(S), run_u, c_ltok, c_token, no_ticket);
 }
 
 __device__ __forceinline__ int hier_walk_row(const CtaRange& cr, int idx) {
@@ -317,7 +347,11 @@ __device__ __forceinline__ int hier_walk_row(const CtaRange& cr, int idx) {
 // loads are issued by the caller before the CTA's first rendezvous (`first_pre`), ahead of the bulk copies' traffic.
 __device__ __forceinline__ void hier_prepare_rows(const StepArgs& a, const CtaRange& cr, const HierTables& tb, int lane,
                                                   int first, int step, const RowPre& first_pre) {
-  const int nq = (a.nblk + 3) >> 2;
+  // the draws belong to block numbers of the whole vocabulary (a shard's first block is number boff); one Philox
+  // call serves the four blocks 4 gq .. 4 gq + 3
+  const int boff = a.vocab_offset >> 10;
+  const int gq0 = boff >> 2;
+  const int nq = ((boff + a.nblk - 1) >> 2) - gq0 + 1;
   for (int g0 = first * 32; g0 < cr.n_local; g0 += step * 32) {
     const int n_g = min(32, cr.n_local - g0);
     if (lane < n_g) {
@@ -332,11 +366,13 @@ __device__ __forceinline__ void hier_prepare_rows(const StepArgs& a, const CtaRa
       if (k >= a.noise_rows) continue;
       const int slot = tb.pre[k].slot, status = tb.pre[k].status, t_now = tb.pre[k].t_now;
       if (slot < 0 || status != ESPO_ROW_ACTIVE) continue;
-      const uint4 rnd = philox4x32_10((uint32_t)q, (uint32_t)t_now, (uint32_t)slot, a.batch_bits | 2u, a.key0, a.key1);
+      const uint4 rnd = philox4x32_10((uint32_t)(gq0 + q), (uint32_t)t_now, (uint32_t)slot, a.batch_bits | 2u, a.key0, a.key1);
       const uint32_t wd[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (4 * q + i < a.nblk) tb.noise[(size_t)k * a.nblk + 4 * q + i] = ln_expo(expo_from_word(wd[i]));
+      for (int i = 0; i < 4; ++i) {
+        const int b = 4 * (gq0 + q) + i - boff;
+        if (b >= 0 && b < a.nblk) tb.noise[(size_t)k * a.nblk + b] = ln_expo(expo_from_word(wd[i]));
+      }
     }
     __syncwarp();
     __threadfence_block();
@@ -381,22 +417,18 @@ __device__ void hier_follow_rows(const StepArgs& a, const CtaRange& cr, const Hi
     const float4* rec = tb.lrec + (k * cr.nblk - cr.b0);            // rec[b] for the CTA's blocks b of the row
     const float* nz = (k < a.noise_rows) ? tb.noise + (size_t)k * a.nblk : nullptr;
     const DrawStream ds{a.key0, a.key1, (uint32_t)pre.t_now, (uint32_t)pre.slot, a.batch_bits};
-    auto noise_at = [&](int b) { return nz ? nz[b] : ln_expo(expo_at(ds, 2u, (uint32_t)b)); };
+    auto noise_at = [&](int b) { return nz ? nz[b] : ln_expo(expo_at(ds, 2u, (uint32_t)(b + (a.vocab_offset >> 10)))); };
     const bool whole = share == a.nblk;
     if (!live) {
       // a row that takes no part needs no records: a whole row is answered at once, a shared one by whoever
       // completes its ticket (every CTA sees the same state, so all of them come here)
       if (whole) {
-        if (pre.slot < 0) mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, true);
-        else mark_row(a, row, pre.slot, lane, -1, 0u, -1, true);
+        hier_skip_row(a, row, lane, pre, true);
       } else {
         unsigned old = 0;
         if (lane == 0) old = atom_add_acq_rel_gpu(a.ticket + row, (unsigned)share);
         old = __shfl_sync(kFullMask, old, 0);
-        if (old + (unsigned)share == (unsigned)a.nblk) {
-          if (pre.slot < 0) mark_row(a, row, 0, lane, -1, ESPO_DEV_BAD_SLOT, -1, false);
-          else mark_row(a, row, pre.slot, lane, -1, 0u, -1, false);
-        }
+        if (old + (unsigned)share == (unsigned)a.nblk) hier_skip_row(a, row, lane, pre, false);
       }
       continue;
     }

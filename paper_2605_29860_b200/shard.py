@@ -52,7 +52,8 @@ def sum_over_ranks(values, dist=None, device="cpu") -> list:
 
 def vocab_shards(V: int, world: int, multiple: int = 128) -> List[Tuple[int, int]]:
     """Contiguous (offset, size) shards of the vocabulary, one per rank; every offset is a multiple of ``multiple``
-    (espo_step_partial wants a multiple of 4; 128 keeps rows of bf16 shards 256-byte aligned).  Trailing ranks may get
+    (espo_step_partial wants a multiple of 4, and of 1024 with the hierarchical sampler, whose draws belong to blocks of
+    1024 ids; 128 keeps rows of bf16 shards 256-byte aligned).  Trailing ranks may get
     an empty shard when V is small."""
     if world < 1 or V < 1 or multiple < 4 or multiple % 4:
         raise ValueError("need world >= 1, V >= 1 and a shard granularity that is a multiple of 4")

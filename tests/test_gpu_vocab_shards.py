@@ -1,5 +1,6 @@
-"""GPU parity of the vocabulary-sharded step (espo_step_partial + espo_step_merge) against the CPU oracle's flat
-sampler on the whole rows, through the C ABI (needs a B200).  The shards of a step are run one after the other on the
+"""GPU parity of the vocabulary-sharded step (espo_step_partial + espo_step_merge) against the CPU oracle's samplers
+on the whole rows, through the C ABI (needs a B200).  The flat sampler's draws belong to token ids, so any cut works;
+the hierarchical sampler's belong to blocks of 1024 ids of the whole vocabulary, so its shards start on one.  The shards of a step are run one after the other on the
 one GPU, which is what N tensor-parallel ranks compute side by side."""
 import numpy as np
 import pytest
@@ -27,14 +28,15 @@ def _sharded_launch(cuts):
     return launch
 
 
+@pytest.mark.parametrize("sampler", [espo.ESPO_SAMPLER_FLAT, espo.ESPO_SAMPLER_HIER])
 @pytest.mark.parametrize("V,world,dtype", [(152064, 8, torch.bfloat16), (152064, 2, torch.float32), (32000, 3, torch.bfloat16),
                                            (5000, 4, torch.float32), (300, 8, torch.bfloat16)])
-def test_sharded_step_matches_the_oracle_on_whole_rows(V, world, dtype):
+def test_sharded_step_matches_the_oracle_on_whole_rows(V, world, dtype, sampler):
     B, T = 24, 6
     p = espo.make_params(temperature=0.8, mu_g=2.0, sigma2_g=4.0, beta=1.5, eps=0.1, t_max=5, eos_token=7,
-                         sampler=espo.ESPO_SAMPLER_FLAT)
+                         sampler=sampler)
     run = ParityRun(B, V, p, seed=77, batch_id=2)
-    run.launch = _sharded_launch(shard.vocab_shards(V, world))
+    run.launch = _sharded_launch(shard.vocab_shards(V, world, multiple=1024 if sampler == espo.ESPO_SAMPLER_HIER else 128))
     for t in range(T):
         x = synth.logits_batch(B, V, dtype=dtype, sd=3.0, seed=900 + t)
         if t == 1:
@@ -74,6 +76,38 @@ def test_cut_does_not_change_the_tokens_and_greedy_takes_the_first_maximum():
     assert torch.all(outs[3] == 123)                        # greedy: the lowest id among equal maxima, across shards
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_hierarchical_shards_give_the_unsharded_tokens(dtype):
+    # the block-level draws are indexed by the block's number in the whole vocabulary, so 1, 2, 3 and 8 shards cut at
+    # multiples of 1024 ids sample exactly the token of espo_step with the hierarchical sampler
+    B, V = 40, 152064
+    v = torch.rand(B, device="cuda")
+    p = espo.make_params(temperature=0.9, mu_g=2.0, sigma2_g=4.0, beta=2.0, t_max=100, sampler=espo.ESPO_SAMPLER_HIER)
+    stop = torch.empty(B, dtype=torch.uint8, device="cuda")
+    for step_seed in (5, 6):
+        x = synth.logits_batch(B, V, dtype=dtype, sd=3.0, seed=step_seed)
+        st2 = espo.espo_init_state(B, V, seed=11)
+        ref_tok = torch.empty(B, dtype=torch.int32, device="cuda")
+        espo.espo_step(x, v, st2, p, ref_tok, stop)
+        ref = {k: a.clone() for k, a in espo.espo_state_view(st2).items()}
+        for world in (1, 2, 3, 8):
+            cuts = shard.vocab_shards(V, world, multiple=1024)
+            st = espo.espo_init_state(B, V, seed=11)
+            tok = torch.empty(B, dtype=torch.int32, device="cuda")
+            parts = torch.empty(len(cuts), B, 8, dtype=torch.float32, device="cuda")
+            for k, (lo, size) in enumerate(cuts):
+                espo.espo_step_partial(x[:, lo:lo + size], lo, st, p, parts[k])
+            espo.espo_step_merge(parts, v, st, p, tok, stop)
+            torch.cuda.synchronize()
+            assert torch.equal(tok, ref_tok), world
+            got = espo.espo_state_view(st)
+            assert torch.equal(got["g"], ref["g"]) and torch.equal(got["status"], ref["status"])
+            assert torch.allclose(got["logp"], ref["logp"], rtol=1e-4, atol=1e-5)
+            assert espo.espo_state_status(st) == 0
+            espo.espo_free_state(st)
+        espo.espo_free_state(st2)
+
+
 def test_argument_errors_of_the_sharded_calls():
     st = espo.espo_init_state(4, 4096, seed=1)
     x = torch.zeros(4, 2048, dtype=torch.bfloat16, device="cuda")
@@ -81,13 +115,15 @@ def test_argument_errors_of_the_sharded_calls():
     flat = espo.make_params(sampler=espo.ESPO_SAMPLER_FLAT)
     hier = espo.make_params(sampler=espo.ESPO_SAMPLER_HIER)
     for kwargs, code in ((dict(off=2, p=flat), espo.ESPO_ERR_BAD_SHAPE), (dict(off=4096, p=flat), espo.ESPO_ERR_BAD_SHAPE),
-                         (dict(off=0, p=hier), espo.ESPO_ERR_BAD_PARAM)):
+                         (dict(off=512, p=hier), espo.ESPO_ERR_BAD_PARAM),        # not on a block of 1024 ids
+                         (dict(off=0, p=espo.make_params(sampler=espo.ESPO_SAMPLER_HIER, temperature=0.0)), espo.ESPO_ERR_BAD_PARAM),
+                         (dict(off=0, p=espo.make_params(sampler=espo.ESPO_SAMPLER_HIER, want_entropy=1)), espo.ESPO_ERR_BAD_PARAM)):
         with pytest.raises(espo.EspoError) as e:
             espo.espo_step_partial(x, kwargs["off"], st, kwargs["p"], parts[0])
         assert e.value.code == code
     with pytest.raises(espo.EspoError) as e:
-        espo.espo_step_merge(parts, torch.zeros(4, device="cuda"), st, hier, torch.empty(4, dtype=torch.int32, device="cuda"),
-                             torch.empty(4, dtype=torch.uint8, device="cuda"))
+        espo.espo_step_merge(parts, torch.zeros(4, device="cuda"), st, espo.make_params(want_entropy=1),
+                             torch.empty(4, dtype=torch.int32, device="cuda"), torch.empty(4, dtype=torch.uint8, device="cuda"))
     assert e.value.code == espo.ESPO_ERR_BAD_PARAM
     espo.espo_free_state(st)
 
