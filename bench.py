@@ -33,7 +33,7 @@ N_BUFFERS = 4                 # 4 x 155.7 MB of logits rotate, so no step finds 
 ADV_B = 1024
 # dram bytes read + written per launch of the step kernel at (B_ROWS, VOCAB, bf16, hierarchical sampler): a constant
 # copied from the ncu capture summarised under profiles/, not measured by this run
-TRAFFIC_STEP_BYTES = 160.6e6
+TRAFFIC_STEP_BYTES = 160.0e6
 TARGET_REGION_MS = 150.0      # short timed regions are repeated until about this much device time has been timed
 
 PARAMS = dict(temperature=1.0, mu_g=6.0, sigma2_g=9.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0, eps=0.2,
@@ -357,7 +357,7 @@ def main():
                      "traffic": TRAFFIC_STEP_BYTES if traffic_known else None,
                      "traffic_source": ("constant from the ncu capture summarised under profiles/ (same kernel, same workload), "
                                         "not measured by this run") if traffic_known else "no capture at this shape",
-                     "kernel": f"espo_step_kernel<bf16,{args.sampler},bulk>",
+                     "kernel": ("espo_step_hier_kernel<bf16,bulk>" if args.sampler == "hier" else "espo_step_kernel<bf16,flat,bulk>"),
                      "peak_kind": f"of {peak_kind} copy bandwidth", "frac_of_nominal_8TBs": achieved / 8000.0,
                      "launch_us": kernel_ms * 1e3, "launch_us_min": stp[0] / K * 1e3, "launch_us_max": stp[-1] / K * 1e3,
                      "bytes_per_launch": bytes_per_launch},
@@ -530,7 +530,16 @@ def main():
                                                             row_ids=ids, n_rows=n_act), N_BUFFERS)
                 act.append({"n_active": n_act, "us": us, "GB/s": n_act * V * 2 / us / 1e3, "rows/s": n_act / (us * 1e-6)})
             ids_out = torch.empty(B, dtype=torch.int32, device=dev)
+
+            def step_then_compact(i):
+                espo.espo_step(bufs[i % N_BUFFERS], values, sst, params, tokens, stop)
+                espo.espo_compact_active(sst, ids_out, n_act_dev)
+            espo.espo_set_dependent_launch(sst, True)
+            pair_us = graph_time_us(step_then_compact, N_BUFFERS)
+            step_alone_us = graph_time_us(lambda i: espo.espo_step(bufs[i % N_BUFFERS], values, sst, params, tokens, stop), N_BUFFERS)
+            espo.espo_set_dependent_launch(sst, False)
             out["active_set"] = {"steps": act,
+                                 "compact_extra_us_dependent_launch": pair_us - step_alone_us,
                                  "compact_us": graph_time_us(lambda i: espo.espo_compact_active(sst, ids_out, n_act_dev), 1),
                                  "note": f"capacity {B} slots, bf16, V={V}; CUDA graphs; compaction is a separate one-CTA kernel"}
             espo.espo_free_state(sst)
@@ -555,7 +564,7 @@ def main():
                 "top_p_0.7_us": step_us(top_p),
                 "top_p_0.9999_us": step_us(top_p_wide),
                 "vocab_shard_partial_us": step_us(flat, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, flat, parts[3]), 16),
-                "vocab_shard_partial_hier_us": step_us(params, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, params, parts[3]), 16),
+                "vocab_shard_partial_hier_us": step_us(hier_params, lambda i, sst: espo.espo_step_partial(shard_bufs[i % 16], lo, sst, hier_params, parts[3]), 16),
                 "vocab_shard_merge_us": step_us(flat, lambda i, sst: espo.espo_step_merge(parts, values, sst, flat, tokens, stop), 1),
                 "note": f"same batch (B={B}, V={V}, bf16), CUDA graphs; partial: one of 8 shards ({n_ids} ids) as its own buffer; "
                         f"merge: 8 x {B} partials",

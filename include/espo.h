@@ -187,7 +187,8 @@ int espo_set_launch_config(espo_state* st, int32_t consumer_warps, int32_t stage
  * GPU may set it up -- place its thread blocks, run the part that touches no global memory -- while the kernel
  * that precedes it in the stream is still finishing; the step kernel waits for that kernel's completion before it
  * reads or writes any global memory, so what it computes does not change.  The step kernel in turn lets a
- * kernel launched after it in the same way start early.  Off by default.  Errors: NULL. */
+ * kernel launched after it in the same way start early; espo_compact_active is launched the same way.  Off by
+ * default.  Errors: NULL. */
 int espo_set_dependent_launch(espo_state* st, int32_t enable);
 
 /* Stable compaction of the active set: writes the slots whose status is ESPO_ROW_ACTIVE, in

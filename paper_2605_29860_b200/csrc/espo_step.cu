@@ -1117,6 +1117,10 @@ __global__ void espo_compact_kernel(const uint8_t* __restrict__ status, int capa
   __shared__ int warp_total[32];
   __shared__ int base;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // (launched as a programmatic dependent when the state asks for it: the step before has completed after the wait;
+  // the kernel after this one may be set up meanwhile)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) base = 0;
   __syncthreads();
   for (int start = 0; start < capacity; start += blockDim.x) {
@@ -1653,8 +1657,15 @@ int espo_state_view(espo_state* st, const float** z, const float** g, const floa
 
 int espo_compact_active(espo_state* st, int32_t* row_ids_out, int32_t* n_active_out, void* stream) {
   if (!st || !row_ids_out || !n_active_out) return ESPO_ERR_NULL;
-  espo::espo_compact_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>(st->status, st->capacity, row_ids_out, n_active_out);
-  ESPO_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(1);
+  cfg.blockDim = dim3(1024);
+  cfg.stream = (cudaStream_t)stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  if (st->dependent_launch) { cfg.attrs = attr; cfg.numAttrs = 1; }
+  ESPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, espo::espo_compact_kernel, (const uint8_t*)st->status, st->capacity, row_ids_out, n_active_out));
   return ESPO_OK;
 }
 
