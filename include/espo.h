@@ -75,6 +75,8 @@ extern "C" {
 #define ESPO_DEV_BAD_ROW     1u   /* some row was marked ESPO_ROW_BAD                       */
 #define ESPO_DEV_BAD_SLOT    2u   /* a row_ids entry was outside [0, capacity)              */
 #define ESPO_DEV_TIMEOUT     4u   /* a bounded in-kernel wait ran out; results incomplete   */
+                                  /* (the launch's row tickets are left stale: call        */
+                                  /* espo_reset_state before the state is used again)      */
 #define ESPO_DEV_NAN_VALUE   8u   /* a value estimate was NaN (that row did not stop)       */
 #define ESPO_DEV_BAD_LENGTHS 16u  /* espo_advantages: sum(lengths) != total_tokens or L < 0 */
 
