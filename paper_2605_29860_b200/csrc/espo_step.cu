@@ -639,10 +639,13 @@ __global__ void __launch_bounds__(64) espo_merge_kernel(const __grid_constant__ 
 constexpr int kFiltThreads = 1024;
 constexpr int kFiltWarps = kFiltThreads / 32;
 constexpr int kFiltSeg = 320;                      // candidate-list entries per warp
-constexpr int kFiltCopies = 16;                    // private copies of the digit histogram (two warps share one)
+constexpr int kFiltCopies = 4;                     // copies of the digit histogram for a candidate list (eight warps share one)
 constexpr int kFiltRing = 4;                       // 16-byte pieces a thread keeps in flight during the pass over the row
 constexpr size_t kFiltRingBytes = (size_t)kFiltRing * kFiltThreads * 16;
+constexpr size_t kFiltLaneHist = (size_t)4 * 256 * 32 * sizeof(unsigned);   // whole-row passes: (3 mass limbs + count) x 256 bins x 32 lanes
 static_assert(kFiltRingBytes >= (size_t)kFiltCopies * 256 * sizeof(uint4), "the histograms reuse the ring's memory");
+static_assert(kFiltRingBytes >= kFiltLaneHist / 2 && (size_t)kFiltWarps * kFiltSeg * sizeof(uint2) >= kFiltLaneHist / 2,
+              "the per-lane histograms reuse the ring's and the candidate list's memory");
 constexpr size_t kFiltSmemBytes = kFiltRingBytes +
                                   256 * (sizeof(unsigned long long) + sizeof(unsigned)) + 192 * sizeof(float) +
                                   (size_t)kFiltWarps * kFiltSeg * (sizeof(uint2) + sizeof(unsigned)) + 128;
@@ -727,6 +730,12 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
   uint2* cand = reinterpret_cast<uint2*>(red_u + 64);                                    // [warps][kFiltSeg] (id, bits)
   unsigned* glist = reinterpret_cast<unsigned*>(cand + kFiltWarps * kFiltSeg);           // [warps][kFiltSeg] first ids of groups with a candidate
   unsigned* sbin = reinterpret_cast<unsigned*>(whist);                                   // 4096 sample bins (before the digit passes)
+  // whole-row digit passes: one copy of every bin per lane, the four limbs in arrays of their own; they reuse the
+  // ring's and the candidate list's memory, both idle by then
+  unsigned* lh0 = reinterpret_cast<unsigned*>(fsm);
+  unsigned* lh1 = lh0 + 256 * 32;
+  unsigned* lh2 = reinterpret_cast<unsigned*>(cand);
+  unsigned* lh3 = lh2 + 256 * 32;
   __shared__ RowPre pre_s;
   __shared__ unsigned long long sh_acc_mass, sh_kept_mass;
   __shared__ unsigned sh_acc_cnt, sh_prefix, sh_cut_a;
@@ -749,8 +758,9 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
 
     const unsigned char* row_base = a.logits + (size_t)row * a.row_stride_bytes;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(row_base) & 15u) == 0;
-    // Calls fn(id, raw bits) for every logit of the row; 16-byte loads where the row allows them.
-    auto for_each = [&](auto&& fn) {
+    // Walks the row (from L2 after the first pass): fnv(first id, four 32-bit words) for every whole 16-byte piece of an
+    // aligned row, fns(id, raw bits) for the logits that are left (all of them if the row is not 16-byte aligned).
+    auto for_each_piece = [&](auto&& fnv, auto&& fns) {
       const int v_main = vec_ok ? (a.V / VEC) * VEC : 0;
       constexpr int kInFlight = 4;                           // loads a thread issues before it looks at the first
       for (int base0 = tid * VEC; base0 < v_main; base0 += kInFlight * kFiltThreads * VEC) {
@@ -765,18 +775,24 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
           const int base = base0 + u * kFiltThreads * VEC;
           if (base >= v_main) break;
           const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (ES == 2) { fn(base + 2 * j, w[j] & 0xffffu); fn(base + 2 * j + 1, w[j] >> 16); }
-            else fn(base + j, w[j]);
-          }
+          fnv(base, w);
         }
       }
       for (int id = v_main + tid; id < a.V; id += kFiltThreads) {
         const uint32_t bits = (ES == 2) ? (uint32_t)__ldg(reinterpret_cast<const unsigned short*>(row_base) + id)
                                         : __ldg(reinterpret_cast<const uint32_t*>(row_base) + id);
-        fn(id, bits);
+        fns(id, bits);
       }
+    };
+    // Calls fn(id, raw bits) for every logit of the row.
+    auto for_each = [&](auto&& fn) {
+      for_each_piece([&](int base, const uint32_t (&w)[4]) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (ES == 2) { fn(base + 2 * j, w[j] & 0xffffu); fn(base + 2 * j + 1, w[j] >> 16); }
+          else fn(base + j, w[j]);
+        }
+      }, fn);
     };
     auto value_of = [&](uint32_t bits) -> float { return __uint_as_float(ES == 2 ? bits << 16 : bits); };
     // The pass over the whole row works on groups of VEC consecutive logits, already as floats: fn(first id,
@@ -979,15 +995,29 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     const unsigned long long kf = a.top_k > 0 ? (unsigned long long)a.top_k : ~0ull;
     const bool use_list = cut_a != 0u && (ma >= pf || ca >= kf) && sh_overflow == 0;
     const bool cut_active = use_list;
-    // Calls fn(id, raw bits) for every logit that can belong to the support.
-    auto for_each_candidate = [&](auto&& fn) {
-      if (use_list) {
-        const unsigned n = seg_n[warp];
-        for (unsigned i = lane; i < n; i += 32) { const uint2 c = my_seg[i]; fn((int)c.x, c.y); }
-      } else {
-        for_each(fn);
+
+    // ---- whole-row search: a first bid for the sampling pass.  The list did not reach top_p or top_k, so each of its
+    //      logits has less than top_p of the mass and fewer than top_k logits above it: all of them stay, and the best
+    //      of their scores is a lower bound of the row's best score (the list's memory is reused below). ----
+    const DrawStream ds{a.key0, a.key1, (uint32_t)pre.t_now, (uint32_t)pre.slot, a.batch_bits};
+    float seed_b = NINF;
+    int seed_id = -1;
+    if (!use_list && cut_a != 0u && sh_overflow == 0) {
+      const unsigned n = seg_n[warp];
+      for (unsigned i = lane; i < n; i += 32) {
+        const uint2 c = my_seg[i];
+        const float x = value_of(c.y);
+        if (!(x > NINF)) continue;
+        const float sc = fmaf(x - M, a.inv_temp, gumbel_at(ds, 0u, c.x));
+        if (sc > seed_b || (sc == seed_b && (int)c.x < seed_id)) { seed_b = sc; seed_id = (int)c.x; }
       }
-    };
+      warp_argmax(seed_b, seed_id);
+      __syncthreads();                                       // red_f of the sums above is no longer read
+      if (lane == 0) { red_f[warp] = seed_b; red_i[warp] = seed_id; }
+      __syncthreads();
+      seed_b = red_f[lane]; seed_id = red_i[lane];
+      warp_argmax(seed_b, seed_id);                          // the same pair in every thread
+    }
 
     // ---- digit passes: find the threshold key.  The keys that take part lie between key_lo (the cut, or 0) and
     //      the key of the largest logit; only the bits in which that range varies are searched, 8 at a time from the
@@ -998,31 +1028,66 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     if (tid == 0) { sh_acc_mass = 0ull; sh_acc_cnt = 0u; sh_prefix = 0u; sh_kept_mass = total; sh_found = 0; }
     for (int d = 0; d < n_digits; ++d) {
       const int shift = 8 * (n_digits - 1 - d);
-      const int copies = use_list ? 4 : kFiltCopies;         // a short list needs few copies, and they cost to clear and add up
-      for (int i = tid; i < copies * 256; i += kFiltThreads) whist[i] = make_uint4(0u, 0u, 0u, 0u);
-      __syncthreads();
-      const uint32_t prefix = sh_prefix;                     // the digits above this one, as found so far
-      unsigned* my_hist = reinterpret_cast<unsigned*>(whist + (warp % copies) * 256);
-      for_each_candidate([&](int, uint32_t bits) {
-        const uint32_t key = filt_key<ES>(bits) - key_lo;    // every candidate's key is at least key_lo
-        if (d > 0 && (key >> (shift + 8)) != prefix) return;
-        const unsigned long long fx = filt_fixed(ex2_approx((value_of(bits) - M) * a.k2));
-        unsigned* h = my_hist + 4u * ((key >> shift) & 255u);
-        atomicAdd(h, (unsigned)(fx >> 26));                  // 14 bits (an e of exactly 1 gives 2^14)
-        atomicAdd(h + 1, (unsigned)(fx >> 13) & 0x1fffu);
-        atomicAdd(h + 2, (unsigned)fx & 0x1fffu);
-        atomicAdd(h + 3, 1u);
-      });
-      __syncthreads();
-      if (tid < 256) {
-        unsigned long long tm = 0ull;
-        unsigned tc = 0u;
-        for (int w = 0; w < copies; ++w) {
-          const uint4 h = whist[w * 256 + tid];
-          tm += ((unsigned long long)h.x << 26) + ((unsigned long long)h.y << 13) + h.z;
-          tc += h.w;
+      if (use_list) {
+        // a short list: four copies of the histogram, one per group of eight warps
+        constexpr int copies = kFiltCopies;
+        for (int i = tid; i < copies * 256; i += kFiltThreads) whist[i] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+        const uint32_t prefix = sh_prefix;                   // the digits above this one, as found so far
+        unsigned* my_hist = reinterpret_cast<unsigned*>(whist + (warp % copies) * 256);
+        const unsigned n = seg_n[warp];
+        for (unsigned i = lane; i < n; i += 32) {
+          const uint32_t bits = my_seg[i].y;
+          const uint32_t key = filt_key<ES>(bits) - key_lo;  // every candidate's key is at least key_lo
+          if (d > 0 && (key >> (shift + 8)) != prefix) continue;
+          const unsigned long long fx = filt_fixed(ex2_approx((value_of(bits) - M) * a.k2));
+          unsigned* h = my_hist + 4u * ((key >> shift) & 255u);
+          atomicAdd(h, (unsigned)(fx >> 26));                // 14 bits (an e of exactly 1 gives 2^14)
+          atomicAdd(h + 1, (unsigned)(fx >> 13) & 0x1fffu);
+          atomicAdd(h + 2, (unsigned)fx & 0x1fffu);
+          atomicAdd(h + 3, 1u);
         }
-        bmass[tid] = tm; bcnt[tid] = tc;
+        __syncthreads();
+        if (tid < 256) {
+          unsigned long long tm = 0ull;
+          unsigned tc = 0u;
+          for (int w = 0; w < copies; ++w) {
+            const uint4 h = whist[w * 256 + tid];
+            tm += ((unsigned long long)h.x << 26) + ((unsigned long long)h.y << 13) + h.z;
+            tc += h.w;
+          }
+          bmass[tid] = tm; bcnt[tid] = tc;
+        }
+      } else {
+        // The whole row: nearly all of its logits fall into a handful of bins, and atomics of one warp on one address
+        // take turns.  So every lane has its own copy of each bin (cell = bin * 32 + lane: the 32 lanes of a warp hit
+        // 32 banks, whatever their bins), shared only with the same lane of the other warps; a cell sees V / 32 logits.
+        for (int i = tid; i < (int)(kFiltLaneHist / 2 / sizeof(uint4)); i += kFiltThreads) {
+          reinterpret_cast<uint4*>(lh0)[i] = make_uint4(0u, 0u, 0u, 0u);
+          reinterpret_cast<uint4*>(lh2)[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncthreads();
+        const uint32_t prefix = sh_prefix;
+        for_each([&](int, uint32_t bits) {
+          const uint32_t key = filt_key<ES>(bits);
+          if (d > 0 && (key >> (shift + 8)) != prefix) return;
+          const unsigned long long fx = filt_fixed(ex2_approx((value_of(bits) - M) * a.k2));
+          const unsigned cell = ((key >> shift) & 255u) * 32u + (unsigned)lane;
+          atomicAdd(lh0 + cell, (unsigned)(fx >> 26));
+          atomicAdd(lh1 + cell, (unsigned)(fx >> 13) & 0x1fffu);
+          atomicAdd(lh2 + cell, (unsigned)fx & 0x1fffu);
+          atomicAdd(lh3 + cell, 1u);
+        });
+        __syncthreads();
+        if (tid < 256) {
+          unsigned long long t0 = 0ull, t1 = 0ull, t2 = 0ull;
+          unsigned tc = 0u;
+          for (int w = 0; w < 32; ++w) {
+            const unsigned cell = (unsigned)tid * 32u + ((unsigned)(w + tid) & 31u);   // the lanes of a warp in 32 banks
+            t0 += lh0[cell]; t1 += lh1[cell]; t2 += lh2[cell]; tc += lh3[cell];
+          }
+          bmass[tid] = (t0 << 26) + (t1 << 13) + t2; bcnt[tid] = tc;
+        }
       }
       __syncthreads();
       if (warp == 0 && (d == 0 || sh_found)) {
@@ -1054,9 +1119,8 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     const unsigned long long kept_mass = sh_kept_mass;
 
     // ---- sampling pass: Gumbel-max over the support with the flat sampler's draws ----
-    const DrawStream ds{a.key0, a.key1, (uint32_t)pre.t_now, (uint32_t)pre.slot, a.batch_bits};
-    float best = NINF;
-    int best_id = -1;
+    float best = seed_b;
+    int best_id = seed_id;
     auto offer = [&](int id, uint32_t bits) {
       if (filt_key<ES>(bits) < tau_key) return;
       const float x = value_of(bits);
@@ -1064,7 +1128,43 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
       const float sc = fmaf(x - M, a.inv_temp, gumbel_at(ds, 0u, (uint32_t)id));
       if (sc > best || (sc == best && id < best_id)) { best = sc; best_id = id; }
     };
-    for_each_candidate(offer);
+    // Four logits whose ids share a Philox counter (id0 is a multiple of 4): one generator call for those that stay.
+    // A logit whose score without noise lies 6 or more under the thread's best needs a Gumbel above 6 to matter; the
+    // draws up to kGumbelBelow6 give less than 5.9001, so they are dropped on the integer and the two logarithms
+    // are taken for one draw in 365 only (the margin of 0.1 covers the rounding of every term many times over).
+    constexpr uint32_t kGumbelBelow6 = 8365658u;             // (2k+1)/2^24 <= exp(-exp(-5.9)) for the 23-bit draw k
+    auto offer4 = [&](int id0, const uint32_t (&b)[4]) {
+      bool in[4];
+      bool any = false;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { in[j] = filt_key<ES>(b[j]) >= tau_key && value_of(b[j]) > NINF; any = any || in[j]; }
+      if (!any) return;
+      const uint4 rnd = philox4x32_10((uint32_t)id0 >> 2, ds.step, ds.slot, ds.batch_bits | 0u, ds.k0, ds.k1);
+      const uint32_t word[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (!in[j]) continue;
+        const float bare = (value_of(b[j]) - M) * a.inv_temp;
+        if (best - bare >= 6.f && (word[j] >> 9) <= kGumbelBelow6) continue;
+        const float sc = fmaf(value_of(b[j]) - M, a.inv_temp, gumbel_from_word(word[j]));
+        if (sc > best || (sc == best && id0 + j < best_id)) { best = sc; best_id = id0 + j; }
+      }
+    };
+    if (use_list) {
+      const unsigned n = seg_n[warp];
+      for (unsigned i = lane; i < n; i += 32) { const uint2 c = my_seg[i]; offer((int)c.x, c.y); }
+    } else {
+      for_each_piece([&](int base, const uint32_t (&w)[4]) {
+        if (ES == 2) {
+          const uint32_t lo[4] = {w[0] & 0xffffu, w[0] >> 16, w[1] & 0xffffu, w[1] >> 16};
+          const uint32_t hi[4] = {w[2] & 0xffffu, w[2] >> 16, w[3] & 0xffffu, w[3] >> 16};
+          offer4(base, lo);
+          offer4(base + 4, hi);
+        } else {
+          offer4(base, w);
+        }
+      }, offer);
+    }
     warp_argmax(best, best_id);
     __syncthreads();                                         // red_f / red_i of the sums above are no longer read
     if (lane == 0) { red_f[warp] = best; red_i[warp] = best_id; }

@@ -57,7 +57,8 @@ def _run_filtered(B, V, dtype, params, steps, seed, make_logits):
 
 
 @pytest.mark.parametrize("V,dtype,top_p,top_k", [(152064, torch.bfloat16, 0.7, 0), (152064, torch.bfloat16, 1.0, 50),
-                                                 (152064, torch.bfloat16, 0.95, 20), (32000, torch.float32, 0.7, 0),
+                                                 (152064, torch.bfloat16, 0.95, 20), (152064, torch.bfloat16, 0.9999, 0),
+                                                 (50001, torch.bfloat16, 0.99, 0), (32000, torch.float32, 0.7, 0),
                                                  (32000, torch.float32, 0.999, 0), (5000, torch.float32, 1.0, 3),
                                                  (777, torch.bfloat16, 0.5, 0), (9, torch.float32, 0.8, 2)])
 def test_filtered_step_matches_the_oracle(V, dtype, top_p, top_k):
