@@ -633,16 +633,19 @@ __global__ void __launch_bounds__(64) espo_merge_kernel(const __grid_constant__ 
 // one threshold tau, which a radix search over the logits' bit patterns finds exactly: one pass per 8-bit digit (two
 // for bfloat16, four for float32), each a histogram of (count, probability mass) over the 256 values of the digit
 // among the logits that share the digits found so far.  Masses are summed as 2^-40 fixed point, so the sums do
-// not depend on the order of the additions and a repeated call takes the same decisions.  One CTA per row; the row
-// is read once from HBM (maximum) and then from L2 (digit passes, sampling pass).
+// not depend on the order of the additions and a repeated call takes the same decisions.  One CTA of 512 threads works
+// on a row at a time, two CTAs share an SM (one's search and sampling fill the gaps of the other's pass); the row is
+// read once from HBM (maximum, candidates) and then, where the candidates do not suffice, from L2 (digit passes,
+// sampling pass).
 // -------------------------------------------------------------------------------------------
-constexpr int kFiltThreads = 1024;
+constexpr int kFiltThreads = 512;                  // two CTAs per SM: one's search and sampling overlap the other's pass over its row
 constexpr int kFiltWarps = kFiltThreads / 32;
-constexpr int kFiltSeg = 320;                      // candidate-list entries per warp
-constexpr int kFiltCopies = 4;                     // copies of the digit histogram for a candidate list (eight warps share one)
+constexpr int kFiltSeg = 400;                      // candidate-list entries per warp
+constexpr int kFiltCopies = 4;                     // copies of the digit histogram for a candidate list (four warps share one)
 constexpr int kFiltRing = 4;                       // 16-byte pieces a thread keeps in flight during the pass over the row
 constexpr size_t kFiltRingBytes = (size_t)kFiltRing * kFiltThreads * 16;
-constexpr size_t kFiltLaneHist = (size_t)4 * 256 * 32 * sizeof(unsigned);   // whole-row passes: (3 mass limbs + count) x 256 bins x 32 lanes
+constexpr int kFiltCells = 16;                     // whole-row passes: copies of every histogram bin (lanes l and l + 16 share one)
+constexpr size_t kFiltLaneHist = (size_t)4 * 256 * kFiltCells * sizeof(unsigned);   // (3 mass limbs + count) x 256 bins x cells
 static_assert(kFiltRingBytes >= (size_t)kFiltCopies * 256 * sizeof(uint4), "the histograms reuse the ring's memory");
 static_assert(kFiltRingBytes >= kFiltLaneHist / 2 && (size_t)kFiltWarps * kFiltSeg * sizeof(uint2) >= kFiltLaneHist / 2,
               "the per-lane histograms reuse the ring's and the candidate list's memory");
@@ -716,7 +719,7 @@ __device__ __forceinline__ FiltCross filt_cross(const unsigned long long* mass, 
 }
 
 template <int ES>
-__global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __grid_constant__ StepArgs a) {
+__global__ void __launch_bounds__(kFiltThreads, 2) espo_filtered_kernel(const __grid_constant__ StepArgs a) {
   extern __shared__ __align__(16) unsigned char fsm[];
   // digit histograms: per bin the mass as three limbs of 14 + 13 + 13 bits (32-bit shared-memory atomics are native,
   // 64-bit ones are not; a copy sees fewer than 2^18 logits per pass, so no limb overflows) and the count
@@ -733,9 +736,9 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
   // whole-row digit passes: one copy of every bin per lane, the four limbs in arrays of their own; they reuse the
   // ring's and the candidate list's memory, both idle by then
   unsigned* lh0 = reinterpret_cast<unsigned*>(fsm);
-  unsigned* lh1 = lh0 + 256 * 32;
+  unsigned* lh1 = lh0 + 256 * kFiltCells;
   unsigned* lh2 = reinterpret_cast<unsigned*>(cand);
-  unsigned* lh3 = lh2 + 256 * 32;
+  unsigned* lh3 = lh2 + 256 * kFiltCells;
   __shared__ RowPre pre_s;
   __shared__ unsigned long long sh_acc_mass, sh_kept_mass;
   __shared__ unsigned sh_acc_cnt, sh_prefix, sh_cut_a;
@@ -843,7 +846,7 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     // ---- candidate cut.  A histogram of the whole row would put nearly every logit into a handful of bins, and
     //      shared-memory atomics on one address serialise.  So 4096 logits (16 stretches of 256 spread over the row)
     //      are sampled into a histogram over the upper 12 bits of their keys, and the cut is the key above which
-    //      64 samples lie -- about 2400 logits of the row.  The pass over the row lists the logits above the cut;
+    //      about 64 samples lie -- about 2400 logits of the row.  The pass over the row lists the logits above the cut;
     //      if they already reach top_p or top_k they contain the whole support and the search below runs over the
     //      list, otherwise (or if the list overflows) it runs over the whole row again. ----
     if (a.V >= 16384) {
@@ -865,12 +868,23 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
         const unsigned long long want = 64ull;
         const FiltCross g = filt_cross(nullptr, bcnt, 0ull, 0u, ~0ull, want, lane);
         if (lane == 0 && g.bin >= 0) {
-          unsigned cum = g.c, edge = (unsigned)(g.bin * 16);
+          // the bin in which the count is reached, and inside it the share of its keys (from the top) that the
+          // missing samples are of the bin's samples: a bin is half a unit wide for logits between 4 and 8, and its
+          // lower edge would admit up to twice the wanted number
+          constexpr int kLow = 8 * ES - 12;                  // key bits below a bin
+          unsigned cum = g.c;
+          unsigned long long cut = (unsigned long long)(g.bin * 16) << kLow;
           for (int i = 15; i >= 0; --i) {
-            cum += sbin[g.bin * 16 + i];
-            if (cum >= want) { edge = (unsigned)(g.bin * 16 + i); break; }
+            const unsigned c = sbin[g.bin * 16 + i];
+            cum += c;
+            if (cum >= want) {
+              const unsigned long long r = want - (cum - c);                          // 1 .. c samples of this bin
+              const unsigned long long take = ((r << kLow) + c - 1) / c;              // 1 .. 2^kLow keys
+              cut = ((unsigned long long)(g.bin * 16 + i + 1) << kLow) - take;
+              break;
+            }
           }
-          sh_cut_a = edge << (8 * ES - 12);                  // the bin's lower edge
+          sh_cut_a = (unsigned)cut;
         }
       }
     }
@@ -963,9 +977,10 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     poisoned = __any_sync(kFullMask, poisoned);
     if (lane == 0) { red_f[warp] = wm; red_i[warp] = poisoned; }
     __syncthreads();
-    static_assert(kFiltWarps == 32, "one lane per warp's partial result");
-    const float M = warp_max(red_f[lane]);                   // every warp folds the 32 partial results by itself
-    poisoned = __any_sync(kFullMask, red_i[lane] != 0);
+    static_assert(kFiltWarps <= 32, "one lane per warp's partial result");
+    const bool has_part = lane < kFiltWarps;
+    const float M = warp_max(has_part ? red_f[lane] : NINF); // every warp folds the warps' partial results by itself
+    poisoned = __any_sync(kFullMask, has_part && red_i[lane] != 0);
     if (poisoned || !(M > NINF)) { mark_row(a, row, pre.slot, tid, 0, ESPO_DEV_BAD_ROW, ESPO_ROW_BAD, true); continue; }
     float tot_f = (m > NINF) ? s_t * ex2_approx((m - M) * a.k2) : 0.f;
     tot_f = warp_sum(tot_f);                                 // fixed order: the same bits on every call
@@ -982,8 +997,8 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     __syncthreads();
     if (lane == 0) { red_f[warp] = tot_f; red_u[warp] = m_a; red_u[32 + warp] = c_a; }
     __syncthreads();
-    double tot = (double)red_f[lane];                        // butterfly: the same tree, hence the same bits, in every lane and call
-    unsigned long long ma = red_u[lane], ca = red_u[32 + lane];   // integer sums: the order does not matter
+    double tot = has_part ? (double)red_f[lane] : 0.0;                        // butterfly: the same tree, hence the same bits, in every lane and call
+    unsigned long long ma = has_part ? red_u[lane] : 0ull, ca = has_part ? red_u[32 + lane] : 0ull;   // integer sums: the order does not matter
 #pragma unroll
     for (int o = 16; o; o >>= 1) {
       tot += __shfl_xor_sync(kFullMask, tot, o);
@@ -1015,7 +1030,7 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
       __syncthreads();                                       // red_f of the sums above is no longer read
       if (lane == 0) { red_f[warp] = seed_b; red_i[warp] = seed_id; }
       __syncthreads();
-      seed_b = red_f[lane]; seed_id = red_i[lane];
+      seed_b = has_part ? red_f[lane] : NINF; seed_id = has_part ? red_i[lane] : -1;
       warp_argmax(seed_b, seed_id);                          // the same pair in every thread
     }
 
@@ -1029,7 +1044,7 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     for (int d = 0; d < n_digits; ++d) {
       const int shift = 8 * (n_digits - 1 - d);
       if (use_list) {
-        // a short list: four copies of the histogram, one per group of eight warps
+        // a short list: four copies of the histogram, one per group of four warps
         constexpr int copies = kFiltCopies;
         for (int i = tid; i < copies * 256; i += kFiltThreads) whist[i] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
@@ -1060,8 +1075,9 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
         }
       } else {
         // The whole row: nearly all of its logits fall into a handful of bins, and atomics of one warp on one address
-        // take turns.  So every lane has its own copy of each bin (cell = bin * 32 + lane: the 32 lanes of a warp hit
-        // 32 banks, whatever their bins), shared only with the same lane of the other warps; a cell sees V / 32 logits.
+        // take turns.  So every bin has kFiltCells copies, picked by the lane (cell = bin * 16 + lane % 16: lanes l and
+        // l + 16 share a cell, the others hit banks of their own whatever their bins); a cell sees V / 16 logits, and
+        // V <= 2^21 keeps the 14-bit limb's sum below 2^31.
         for (int i = tid; i < (int)(kFiltLaneHist / 2 / sizeof(uint4)); i += kFiltThreads) {
           reinterpret_cast<uint4*>(lh0)[i] = make_uint4(0u, 0u, 0u, 0u);
           reinterpret_cast<uint4*>(lh2)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -1072,7 +1088,7 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
           const uint32_t key = filt_key<ES>(bits);
           if (d > 0 && (key >> (shift + 8)) != prefix) return;
           const unsigned long long fx = filt_fixed(ex2_approx((value_of(bits) - M) * a.k2));
-          const unsigned cell = ((key >> shift) & 255u) * 32u + (unsigned)lane;
+          const unsigned cell = ((key >> shift) & 255u) * (unsigned)kFiltCells + ((unsigned)lane & (kFiltCells - 1));
           atomicAdd(lh0 + cell, (unsigned)(fx >> 26));
           atomicAdd(lh1 + cell, (unsigned)(fx >> 13) & 0x1fffu);
           atomicAdd(lh2 + cell, (unsigned)fx & 0x1fffu);
@@ -1082,8 +1098,8 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
         if (tid < 256) {
           unsigned long long t0 = 0ull, t1 = 0ull, t2 = 0ull;
           unsigned tc = 0u;
-          for (int w = 0; w < 32; ++w) {
-            const unsigned cell = (unsigned)tid * 32u + ((unsigned)(w + tid) & 31u);   // the lanes of a warp in 32 banks
+          for (int w = 0; w < kFiltCells; ++w) {
+            const unsigned cell = (unsigned)tid * kFiltCells + ((unsigned)(w + tid) & (kFiltCells - 1));   // the lanes of a warp spread over the banks
             t0 += lh0[cell]; t1 += lh1[cell]; t2 += lh2[cell]; tc += lh3[cell];
           }
           bmass[tid] = (t0 << 26) + (t1 << 13) + t2; bcnt[tid] = tc;
@@ -1170,8 +1186,8 @@ __global__ void __launch_bounds__(kFiltThreads, 1) espo_filtered_kernel(const __
     if (lane == 0) { red_f[warp] = best; red_i[warp] = best_id; }
     __syncthreads();
     if (warp == 0) {
-      float b = red_f[lane];
-      int tok = red_i[lane];
+      float b = has_part ? red_f[lane] : NINF;
+      int tok = has_part ? red_i[lane] : -1;
       warp_argmax(b, tok);                                   // largest score, the smaller id among equal ones, -1 if none
       if (lane == 0) {
         if (tok < 0) {
@@ -1578,11 +1594,11 @@ static int step_launch(const void* logits, int32_t logits_dtype, int64_t row_str
   a.tokens_out = tokens_out; a.stop_out = stop_out;
 
   if (!a.greedy && (a.top_p < 1.f || a.top_k > 0)) {
-    // filtered sampling: its own kernel, one CTA per row
+    // filtered sampling: its own kernel, one CTA per row at a time, two CTAs per SM
     if (p->sampler != ESPO_SAMPLER_FLAT || partial_out) return ESPO_ERR_BAD_PARAM;
     if (v_eff > (1 << 21)) return ESPO_ERR_CAPACITY;       // the histogram limbs are sized for rows up to 2^21 logits
     auto fk = (es == 2) ? espo_filtered_kernel<2> : espo_filtered_kernel<4>;
-    const int fgrid = n_rows < st->sm_count ? n_rows : st->sm_count;
+    const int fgrid = n_rows < 2 * st->sm_count ? n_rows : 2 * st->sm_count;
     fk<<<(unsigned)fgrid, kFiltThreads, kFiltSmemBytes, (cudaStream_t)stream>>>(a);
     ESPO_CUDA_TRY(cudaGetLastError());
     return ESPO_OK;
