@@ -38,6 +38,7 @@ TARGET_REGION_MS = 250.0      # short timed regions are repeated until about thi
 
 PARAMS = dict(temperature=1.0, mu_g=6.0, sigma2_g=9.0, delta=1e-8, clip_c=10.0, alpha_s=0.9, beta=7.0, eps=0.2,
               warmup_complete=1, t_max=1 << 30, eos_token=-1)
+FILTER = {}   # top_p / top_k of the timed step when --top-p / --top-k ask for the filtered step
 
 
 def measured_peaks():
@@ -125,7 +126,7 @@ def oracle_step_rate(rows_f32, values, seconds_target: float, sampler: int, core
     """
     import oracle
     cores = cores or cpu_threads()
-    p = oracle.make_params(sampler=sampler, **PARAMS)
+    p = oracle.make_params(sampler=sampler, **PARAMS, **FILTER)
     n = rows_f32.shape[0]
     ro = oracle.Rollout(n, seed=1)
     done, t0 = 0, time.perf_counter()
@@ -192,6 +193,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=B_ROWS, help="rollout batch size B (default: the headline 512)")
     ap.add_argument("--sampler", default="hier", choices=["hier", "flat"])
+    ap.add_argument("--top-p", type=float, default=1.0, help="time the filtered step instead (needs --sampler flat)")
+    ap.add_argument("--top-k", type=int, default=0, help="time the filtered step instead (needs --sampler flat)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the single-step timings at other shapes")
     ap.add_argument("--eager", action="store_true", help="launch every step separately instead of replaying a CUDA graph")
@@ -226,7 +229,12 @@ def main():
 
     B, V, K, W = args.rows, VOCAB, args.steps, args.warmup
     sampler = espo.ESPO_SAMPLER_HIER if args.sampler == "hier" else espo.ESPO_SAMPLER_FLAT
-    params = espo.make_params(sampler=sampler, **PARAMS)
+    filtered = args.top_p < 1.0 or args.top_k > 0
+    if filtered:
+        if args.sampler != "flat":
+            raise SystemExit("--top-p / --top-k need --sampler flat (the filtered step draws with the flat sampler)")
+        FILTER.update(top_p=args.top_p, top_k=args.top_k)
+    params = espo.make_params(sampler=sampler, **PARAMS, **FILTER)
     # ---- synthetic inputs, resident in HBM: every rank owns its own B rows (rows are independent) ----
     plan = shard.rank_plan(rank, world, B)
     bufs = [synth.logits_batch(B, V, dtype=torch.bfloat16, sd=3.0, seed=100 + plan["data_seed_offset"] + i, device=dev)
@@ -341,7 +349,9 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": f"rollout-batch scale: B={B} trajectories per GPU, V={V}, bf16 logits ~N(0,3) + 5 Zipf peaks, "
-                        f"temperature 1.0, {args.sampler} Philox Gumbel-max sampler, full active set; timed region = "
+                        f"temperature 1.0, {args.sampler} Philox Gumbel-max sampler"
+                        + (f" over the top-p {args.top_p} / top-k {args.top_k} support" if filtered else "")
+                        + f", full active set; timed region = "
                         f"{K} decode steps + 1 advantage pass over the {adv_tokens} tokens generated",
             "logits_dtype": "bf16", "arithmetic": "f32 (f64 for the advantage scan's composition)",
             "launch": ("eager launches" if graph is None else f"CUDA graph of {graph_steps} steps, replayed once before timing")
@@ -359,7 +369,8 @@ def main():
                      "traffic": TRAFFIC_STEP_BYTES if traffic_known else None,
                      "traffic_source": ("constant from the ncu capture summarised under profiles/ (same kernel, same workload), "
                                         "not measured by this run") if traffic_known else "no capture at this shape",
-                     "kernel": ("espo_step_hier_kernel<bf16,bulk>" if args.sampler == "hier" else "espo_step_kernel<bf16,flat,bulk>"),
+                     "kernel": ("espo_filtered_kernel<bf16>" if filtered else "espo_step_hier_kernel<bf16,bulk>" if args.sampler == "hier"
+                                else "espo_step_kernel<bf16,flat,bulk>"),
                      "peak_kind": f"of {peak_kind} copy bandwidth", "frac_of_nominal_8TBs": achieved / 8000.0,
                      "launch_us": kernel_ms * 1e3, "launch_us_min": stp[0] / K * 1e3, "launch_us_max": stp[-1] / K * 1e3,
                      "bytes_per_launch": bytes_per_launch},
