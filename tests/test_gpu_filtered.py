@@ -59,6 +59,8 @@ def _run_filtered(B, V, dtype, params, steps, seed, make_logits):
 @pytest.mark.parametrize("V,dtype,top_p,top_k", [(152064, torch.bfloat16, 0.7, 0), (152064, torch.bfloat16, 1.0, 50),
                                                  (152064, torch.bfloat16, 0.95, 20), (152064, torch.bfloat16, 0.9999, 0),
                                                  (50001, torch.bfloat16, 0.99, 0), (32000, torch.float32, 0.7, 0),
+                                                 (152064, torch.float32, 0.999, 0), (152064, torch.bfloat16, 1.0, 5000),
+                                                 (16391, torch.bfloat16, 0.97, 0), (16391, torch.bfloat16, 0.6, 0),
                                                  (32000, torch.float32, 0.999, 0), (5000, torch.float32, 1.0, 3),
                                                  (777, torch.bfloat16, 0.5, 0), (9, torch.float32, 0.8, 2)])
 def test_filtered_step_matches_the_oracle(V, dtype, top_p, top_k):
@@ -105,3 +107,28 @@ def test_support_is_respected_and_ties_stay_together():
     assert e.value.code == espo.ESPO_ERR_BAD_PARAM
     for s in (st, st2, st3):
         espo.espo_free_state(s)
+
+
+def test_more_tied_candidates_than_the_list_holds():
+    # 10 000 equal logits at the top key of a sample-histogram bin: all of them lie above the candidate cut, the list
+    # overflows, and the search runs over the whole row; top_k = 2 keeps exactly the tied tokens
+    B, V, n_top = 8, 40000, 10000
+    x = torch.full((B, V), -3.0, dtype=torch.bfloat16, device="cuda")
+    g = torch.Generator().manual_seed(11)
+    top_val = torch.tensor([0x408F], dtype=torch.int16).view(torch.bfloat16).item()     # 4.46875: low key bits 1111
+    heavy = [torch.randperm(V, generator=g)[:n_top].cuda() for _ in range(B)]
+    for r in range(B):
+        x[r, heavy[r]] = top_val
+    p = espo.make_params(temperature=1.0, sampler=espo.ESPO_SAMPLER_FLAT, top_k=2, beta=1e9, t_max=10**6)
+    st = espo.espo_init_state(B, V, seed=21)
+    tok = torch.empty(B, dtype=torch.int32, device="cuda"); stop = torch.empty(B, dtype=torch.uint8, device="cuda")
+    v = torch.zeros(B, device="cuda")
+    for _ in range(6):
+        espo.espo_step(x, v, st, p, tok, stop)
+        torch.cuda.synchronize()
+        assert espo.espo_state_status(st) == 0
+        lp = espo.espo_state_view(st)["logp"].cpu().numpy()
+        assert np.allclose(lp, -np.log(n_top), atol=1e-5)
+        for r in range(B):
+            assert float(x[r, int(tok[r])]) == top_val
+    espo.espo_free_state(st)
