@@ -515,6 +515,7 @@ def main():
                         nb = max(2, int(280e6 // per) + 1)
                         sbufs = [synth.logits_batch(sB, sV, dtype=sdt, sd=3.0, seed=500 + i, device=dev) for i in range(nb)]
                         sst = espo.espo_init_state(sB, sV, seed=99)
+                        espo.espo_set_dependent_launch(sst, use_pdl)      # the main region's launch mode
                         sval = torch.full((sB,), 0.5, dtype=torch.bfloat16, device=dev)
                         stok = torch.empty(sB, dtype=torch.int32, device=dev)
                         sstop = torch.empty(sB, dtype=torch.uint8, device=dev)
@@ -529,12 +530,15 @@ def main():
                         del sbufs
             out["bandwidth_sweep"] = {"shapes": sweep,
                                       "note": "one espo_step per launch, CUDA graph of >= 40 launches over rotating buffers "
-                                              "(> 280 MB in total), full active set; GB/s = B*V*sizeof(logit) / time"}
+                                              "(> 280 MB in total), full active set; GB/s = B*V*sizeof(logit) / time; "
+                                              + ("hierarchical step launched as a programmatic dependent, like the main region"
+                                                 if use_pdl else "plain launches")}
 
             # ---- shrinking active set: as rows stop, the caller passes the n_active surviving rows (compacted
             #      logits plus the slot list from espo_compact_active); per-step time vs n_active ----
             act = []
             sst = espo.espo_init_state(B, V, seed=7)
+            espo.espo_set_dependent_launch(sst, use_pdl)
             all_ids = torch.arange(B, dtype=torch.int32, device=dev)
             n_act_dev = torch.zeros(1, dtype=torch.int32, device=dev)
             for n_act in (B, (3 * B) // 4, B // 2, B // 4, B // 8):
@@ -554,13 +558,16 @@ def main():
             out["active_set"] = {"steps": act,
                                  "compact_extra_us_dependent_launch": pair_us - step_alone_us,
                                  "compact_us": graph_time_us(lambda i: espo.espo_compact_active(sst, ids_out, n_act_dev), 1),
-                                 "note": f"capacity {B} slots, bf16, V={V}; CUDA graphs; compaction is a separate one-CTA kernel"}
+                                 "note": f"capacity {B} slots, bf16, V={V}; CUDA graphs, "
+                                         + ("step launched as a programmatic dependent" if use_pdl else "plain launches")
+                                         + "; compaction is a separate one-CTA kernel"}
             espo.espo_free_state(sst)
 
         # ---- the other routes through the step: flat sampler, top-p filter, vocabulary shards ----
         if not args.no_sweep:
             def step_us(p, fn=None, n_var=N_BUFFERS):
                 sst = espo.espo_init_state(B, V, seed=5)
+                espo.espo_set_dependent_launch(sst, use_pdl)          # (only the hierarchical kernels are launched that way)
                 call = (lambda i: espo.espo_step(bufs[i % N_BUFFERS], values, sst, p, tokens, stop)) if fn is None else (lambda i: fn(i, sst))
                 us = graph_time_us(call, n_var)
                 espo.espo_free_state(sst)

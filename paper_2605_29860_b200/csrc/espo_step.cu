@@ -1493,6 +1493,21 @@ static int launch_hier(espo::StepArgs& a, const espo_state* st, int es, bool bul
   a.blk_base = (int)(a.total_blocks / grid);
   a.blk_rem = (int)(a.total_blocks % grid);
   const long long blocks_per_cta = (a.total_blocks + grid - 1) / grid;
+  if (!st->cfg_warps && es == 2) {
+    // The launch ends when the warp with the most blocks ends, and the warps share the SM's transcendental pipe, so
+    // what counts is blocks per warp (rounded up) x warps: a range of 516 blocks costs 30 warps 18 x 30 = 540 block
+    // times and 26 warps 20 x 26 = 520 (measured at B=512, V=152064: 30.5 against 29.9 us).  Warps are taken away four
+    // at a time, so that the SM's four schedulers keep equal numbers (28 or 24 streaming warps measured worse than
+    // either neighbour), and every warp less costs about 0.3 % of throughput in latency hiding (at B=2048 thirty
+    // warps win).
+    int best_w = warps;
+    long long best_cost = -1;
+    for (int w = warps; w >= warps - 8 && w >= 8; w -= 4) {
+      const long long cost = (blocks_per_cta + w - 1) / w * w * (1000 + 3 * (warps - w));
+      if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_w = w; }
+    }
+    warps = best_w;
+  }
   if (blocks_per_cta < warps) warps = (int)blocks_per_cta;
   const long long rows = blocks_per_cta / a.nblk + 2;      // rows a CTA's range can touch
   if (rows > kMaxQueue) return 1;
