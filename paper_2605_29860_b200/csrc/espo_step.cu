@@ -1495,15 +1495,17 @@ static int launch_hier(espo::StepArgs& a, const espo_state* st, int es, bool bul
   const long long blocks_per_cta = (a.total_blocks + grid - 1) / grid;
   if (!st->cfg_warps && es == 2) {
     // The launch ends when the warp with the most blocks ends, and the warps share the SM's transcendental pipe, so
-    // what counts is blocks per warp (rounded up) x warps: a range of 516 blocks costs 30 warps 18 x 30 = 540 block
-    // times and 26 warps 20 x 26 = 520 (measured at B=512, V=152064: 30.5 against 29.9 us).  Warps are taken away four
-    // at a time, so that the SM's four schedulers keep equal numbers (28 or 24 streaming warps measured worse than
-    // either neighbour), and every warp less costs about 0.3 % of throughput in latency hiding (at B=2048 thirty
-    // warps win).
+    // the sweep costs blocks per warp (rounded up) x warps block times of about 0.046 us: a range of 516 blocks costs
+    // 30 warps 18 x 30 = 540 of them and 26 warps 20 x 26 = 520 (measured at B=512, V=152064: 30.5 against 29.9 us).
+    // Warps are taken away four at a time, so that the SM's four schedulers keep equal numbers (28 or 24 streaming
+    // warps measured worse than either neighbour).  Every warp less costs about 0.5 % of streaming throughput
+    // (latency hiding: at B=2048 thirty warps win) and saves 0.04 us of fixed time per launch, 0.1 us when the
+    // launch is a programmatic dependent (fitted to launches of 64 to 2048 rows: 22 warps win below 256 rows).
+    const long long per_warp_fixed = st->dependent_launch ? 2174 : 870;    // in units of 1/1000 block time
     int best_w = warps;
     long long best_cost = -1;
     for (int w = warps; w >= warps - 8 && w >= 8; w -= 4) {
-      const long long cost = (blocks_per_cta + w - 1) / w * w * (1000 + 3 * (warps - w));
+      const long long cost = (blocks_per_cta + w - 1) / w * w * (1000 + 5 * (warps - w)) + per_warp_fixed * w;
       if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_w = w; }
     }
     warps = best_w;
