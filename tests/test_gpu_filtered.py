@@ -132,3 +132,21 @@ def test_more_tied_candidates_than_the_list_holds():
         for r in range(B):
             assert float(x[r, int(tok[r])]) == top_val
     espo.espo_free_state(st)
+
+
+@pytest.mark.parametrize("V,dtype,top_p,top_k", [(152064, torch.bfloat16, 0.7, 0), (20480, torch.bfloat16, 0.9999, 0),
+                                                 (16384, torch.float32, 0.6, 0), (50008, torch.bfloat16, 1.0, 40)])
+def test_more_rows_than_ctas(V, dtype, top_p, top_k):
+    # 330 rows on 296 CTAs: some CTAs work through two rows one after the other (shared-memory lists and histograms reused)
+    B, T = 330, 3
+    p = espo.make_params(temperature=0.9, mu_g=2.0, sigma2_g=4.0, beta=1.5, eps=0.1, t_max=4, eos_token=3,
+                         sampler=espo.ESPO_SAMPLER_FLAT, top_p=top_p, top_k=top_k)
+    def logits(t):
+        x = synth.logits_batch(B, V, dtype=dtype, sd=2.5, seed=140 + t)
+        if t == 1:
+            x[1, : V // 3] = float("-inf")                  # masked ids
+            x[2, 7] = float("nan")                          # an unusable row
+            x[5, V - 1] = float("inf")                      # another one
+        return x
+    checked, excused, ties = _run_filtered(B, V, dtype, p, T, seed=13, make_logits=logits)
+    assert checked >= 2 * B and excused <= 8 and ties <= 5, (checked, excused, ties)
