@@ -900,22 +900,42 @@ __global__ void __launch_bounds__(kFiltThreads, 2) espo_filtered_kernel(const __
                                       : value_of((cut_a & key_top) ? (cut_a & ~key_top) : (~cut_a & (ES == 2 ? 0xffffu : 0xffffffffu)));
 
     // ---- the pass over the row (from HBM): the largest logit and the row's mass sum_a exp((x_a - M)/T), kept per
-    //      thread relative to the thread's own running maximum; NaN or +inf anywhere makes the row unusable (either
-    //      turns the thread's sum into NaN or its maximum into +inf); logits at or above the cut go onto the list. ----
+    //      lane relative to the warp's running maximum; NaN or +inf anywhere makes the row unusable (either turns a
+    //      lane's sum into NaN or the maximum into +inf); logits at or above the cut go onto the list. ----
     float m = NINF, s_t = 0.f;
     uint2* my_seg = cand + warp * kFiltSeg;
     unsigned* my_groups = glist + warp * kFiltSeg;
+    // The warp keeps one running maximum mw for all of its lanes (a trip's maximum comes from one redux), so that the
+    // exponents are one packed multiply-add x*k2 + c0 with c0 = -mw*k2 and the sums packed adds; c0 is rounded once
+    // per value of mw, which leaves every term of that stretch with the common factor 2^dl, dl = c0 + mw*k2 (exact
+    // as a fused multiply-add), taken out when mw moves and at the end.
+    float mw = NINF, c0 = 0.f;
+    float2 acc = make_float2(0.f, 0.f);
+    bool nan_seen = false;
     for_each_group([&](int base, const float (&x)[VEC]) {
       float vm = x[0];
 #pragma unroll
       for (int j = 1; j < VEC; ++j) vm = fmaxf(vm, x[j]);
-      if (vm > m) { s_t *= ex2_approx((m - vm) * a.k2); m = vm; }   // m = -inf: s_t is 0 and stays 0
-      if (m > NINF) {
+      const float wmax = warp_max(vm);
+      if (wmax > mw) {                                       // the same in every lane
+        if (mw > NINF) {
+          const float dl = fmaf(mw, a.k2, c0);
+          const float sc = ex2_approx(fmaf(mw - wmax, a.k2, -dl));   // to the new maximum, the old stretch's factor out
+          acc.x *= sc; acc.y *= sc;
+        }
+        mw = wmax;
+        c0 = -mw * a.k2;
+      }
+      if (mw > NINF) {
+        const float2 k2v = make_float2(a.k2, a.k2), c0v = make_float2(c0, c0);
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) s_t += ex2_approx((x[j] - m) * a.k2);     // NaN stays NaN; +inf makes m +inf, then NaN
+        for (int j = 0; j < VEC / 2; ++j) {                  // NaN stays NaN; +inf makes mw +inf, then NaN or 0
+          const float2 t = __ffma2_rn(make_float2(x[2 * j], x[2 * j + 1]), k2v, c0v);
+          acc = __fadd2_rn(acc, make_float2(ex2_approx(t.x), ex2_approx(t.y)));
+        }
       } else {
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) if (x[j] != x[j]) s_t = x[j];             // a NaN among logits that are all -inf so far
+        for (int j = 0; j < VEC; ++j) nan_seen = nan_seen || (x[j] != x[j]);   // a NaN among logits that are all -inf so far
       }
       // About one logit in 50 lies above the cut, so in nearly every trip some lane of the warp has one, and what the
       // lane does about it the whole warp waits for: the pass only notes the group on the warp's list of groups
@@ -926,6 +946,10 @@ __global__ void __launch_bounds__(kFiltThreads, 2) espo_filtered_kernel(const __
         else sh_overflow = 1;
       }
     });
+    m = mw;
+    s_t = (acc.x + acc.y) * ex2_approx(-fmaf(mw, a.k2, c0));
+    if (!(mw > NINF)) s_t = 0.f;
+    if (nan_seen) s_t = __int_as_float(0x7fc00000);
     // ---- the noted groups, read again (L2, a few per lane), give the list of candidates ----
     __syncwarp();
     {
